@@ -1,0 +1,95 @@
+/*
+ * CPU oracle for the FeF-DLLM speculative-verification step.
+ *
+ * TEST INFRASTRUCTURE ONLY. This is a plain, slow, single-threaded,
+ * double-precision restatement of what the paper's decoding algorithm
+ * computes per speculative window (Algorithm 2, inner verification loop;
+ * the residual law of Eq. "residual_distribution_alg"; Section 3.2), and of
+ * the LowConf selection of Algorithm 2.  It shares no code, header, table or
+ * constant generator with the CUDA library and neither includes the other.
+ * Only tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+ *
+ * All pointers are HOST pointers.  Layouts match the CUDA library's so the
+ * same bytes can be given to both.
+ *
+ * Pins (tests/test_oracle_pins.py): Philox against the cuRAND host generator,
+ * softmax against a float64 library softmax, acceptance probability
+ * = sum_z min(pi, rho), emitted-token law = pi by exact enumeration and by
+ * chi-square, p = q accepts everything, residual sums to one, mean committed
+ * length = sum_l prod_{i<l} alpha_i (Theorem 2 when the alpha_i are equal),
+ * LowConf against a library stable sort.
+ * Parity unpinned by the paper (readings fixed by this build only): the
+ * confidence reported at temperature 0, tie order in LowConf, sentinel values
+ * beyond the committed prefix.
+ */
+#ifndef FEF_ORACLE_H
+#define FEF_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status values (numerically the same meaning as the library's, restated) */
+enum {
+    FEFO_OK = 0,
+    FEFO_ERR_INVALID_ARG = 1,
+    FEFO_ERR_DTYPE = 2,
+    FEFO_ERR_NONFINITE = 7,
+    FEFO_ERR_TOKEN_RANGE = 8
+};
+
+/* logit storage types */
+enum { FEFO_F32 = 0, FEFO_BF16 = 1 };
+
+/* Philox4x32-10 block function: out[4] = philox(ctr[4], key[2]). */
+void fef_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+
+/* The uniform the verification step draws.
+ * key = (low 32 bits of seed, high 32 bits of seed);
+ * counter = ((stream << 30) | j, b, pos, step); the `lane`-th output word r
+ * maps to u = ((r >> 9) + 0.5) * 2^-23, which lies strictly inside (0, 1). */
+double fef_oracle_uniform(uint64_t seed, uint32_t stream, uint32_t j, uint32_t b,
+                          uint32_t pos, uint32_t step, uint32_t lane);
+
+/* Laws of ONE position (Section 3.2): pi = softmax(p_logits / T),
+ * rho = softmax(q_logits / T), resid = [pi - rho]_+ / (1 - sum_z min(pi, rho))
+ * (all zeros when that denominator is 0), *alpha = sum_z min(pi, rho).
+ * T must be > 0.  Returns a status. */
+int fef_oracle_row_laws(const void* p_logits, const void* q_logits, int V, int dtype,
+                        float temperature, double* pi, double* rho, double* resid,
+                        double* alpha);
+
+/* One verification call over B independent windows of K positions
+ * (Algorithm 2, the loop "for m = 1..b").
+ *   draft_logits, target_logits : [B, K, ld] (ld >= V), dtype F32 or BF16
+ *   draft_tokens                : [B, K]
+ *   row_len                     : [B] number of valid drafts (0..K), or NULL = K
+ *   temperature                 : > 0 sampling; == 0 greedy (see DESIGN notes in
+ *                                 the .cpp); < 0 invalid
+ * Outputs (caller allocated):
+ *   accept_len [B]    index of first rejected draft, or row_len if none; -1 on a data error
+ *   tokens     [B, K] committed tokens (accepted drafts, then the corrected token); -1 beyond
+ *   conf       [B, K] double; pi(committed token); -1 beyond
+ *   accept_margin [B, K] (may be NULL) |u - pi(x)/rho(x)| of every acceptance test made, else +inf
+ *   gumbel_gap    [B]    (may be NULL) best minus second-best Gumbel score of the
+ *                        residual draw, +inf when no draw or a single candidate
+ * Returns the largest status over the batch rows. */
+int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
+                           const int32_t* draft_tokens, const int32_t* row_len,
+                           int B, int K, int V, int64_t ld, int dtype,
+                           float temperature, uint64_t seed, uint32_t step,
+                           int32_t* accept_len, int32_t* tokens, double* conf,
+                           double* accept_margin, double* gumbel_gap);
+
+/* LowConf_k (Algorithm 2): per batch row the k candidates (mask != 0) of lowest
+ * confidence, ordered by (conf ascending, index ascending).
+ *   conf [B, L] float, mask [B, L] uint8 -> positions [B, k] (-1 padded), count [B]. */
+int fef_oracle_remask_select(const float* conf, const uint8_t* mask, int B, int L, int k,
+                             int32_t* positions, int32_t* count);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

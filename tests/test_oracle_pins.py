@@ -1,0 +1,533 @@
+"""The CPU oracle against what the paper and the mathematics fix (no GPU).
+
+Every check compares the oracle with something other than itself: a library
+routine (cuRAND's host Philox generator, torch's float64 softmax, numpy's stable
+sort), a closed form from the paper, an exact enumeration, or a statistical law.
+"""
+import ctypes
+import glob
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------- helpers ----
+def _f32(a):
+    return torch.tensor(np.asarray(a, dtype=np.float32))
+
+
+def _softmax64(logits, T=1.0):
+    return torch.softmax(torch.as_tensor(np.asarray(logits), dtype=torch.float64) / T, dim=-1).numpy()
+
+
+def _draw_from(prob, n, rng):
+    """n iid draws from a small categorical law with numpy's generator (inverse cdf)."""
+    cdf = np.cumsum(prob)
+    cdf[-1] = 1.0
+    return np.searchsorted(cdf, rng.random(n), side="right").astype(np.int32)
+
+
+def _tile(row, B, K=1):
+    """[V] or [K,V] logits -> [B,K,V] float32 tensor."""
+    r = np.asarray(row, dtype=np.float32)
+    if r.ndim == 1:
+        r = r[None, :]
+    return _f32(np.broadcast_to(r[None], (B,) + r.shape).copy())
+
+
+# ------------------------------------------------------------------ Philox ----
+def _curand():
+    cands = ["/usr/local/cuda/lib64/libcurand.so.10", "libcurand.so.10"]
+    cands += glob.glob(os.path.join(os.path.dirname(torch.__file__), "..", "nvidia", "curand", "lib", "libcurand.so*"))
+    for c in cands:
+        try:
+            return ctypes.CDLL(c)
+        except OSError:
+            continue
+    return None
+
+
+def _curand_host_philox(lib, seed, offset, n):
+    gen = ctypes.c_void_p()
+    assert lib.curandCreateGeneratorHost(ctypes.byref(gen), 161) == 0  # CURAND_RNG_PSEUDO_PHILOX4_32_10
+    assert lib.curandSetPseudoRandomGeneratorSeed(gen, ctypes.c_ulonglong(seed)) == 0
+    assert lib.curandSetGeneratorOffset(gen, ctypes.c_ulonglong(offset)) == 0
+    out = np.zeros(n, dtype=np.uint32)
+    assert lib.curandGenerate(gen, out.ctypes.data_as(ctypes.c_void_p), ctypes.c_size_t(n)) == 0
+    lib.curandDestroyGenerator(gen)
+    return out
+
+
+def test_philox_matches_curand_host_generator():
+    """cuRAND's host Philox4_32_10 generator interleaves 65536 subsequences: its
+    4-word block number i holds philox(counter = (i // 65536 [64-bit, words 0-1],
+    i % 65536 [word 2], 0), key = seed).  That pins the round function, the
+    multipliers, the key schedule, the round count and the key/seed split."""
+    lib = _curand()
+    if lib is None:
+        pytest.skip("libcurand not loadable")
+    for seed in (0, 0x123456789ABCDEF0, 0xFFFFFFFFFFFFFFFF):
+        key = [seed & 0xFFFFFFFF, seed >> 32]
+        # plain start: counters (0..1, 0, 0..65535, 0)
+        out = _curand_host_philox(lib, seed, 0, 4 * 65536 * 2).reshape(-1, 4)
+        for blk in list(range(0, 300)) + [65535, 65536, 65537, 131071]:
+            ctr = [blk // 65536, 0, blk % 65536, 0]
+            assert (oracle.philox4x32_10(ctr, key) == out[blk]).all(), (seed, blk)
+        # large offset: carries through word 0 into word 1
+        c0, c1 = 0xFFFFFFFE, 0x1234
+        off = 4 * 65536 * ((c1 << 32) | c0) + 4 * 77
+        out = _curand_host_philox(lib, seed, off, 4 * 65536 * 2 + 4 * 80).reshape(-1, 4)
+        for blk, ctr in [(0, [c0, c1, 77, 0]), (1, [c0, c1, 78, 0]), (65536 - 77, [c0 + 1, c1, 0, 0]),
+                         (2 * 65536 - 77, [0, c1 + 1, 0, 0]), (2 * 65536, [0, c1 + 1, 77, 0])]:
+            assert (oracle.philox4x32_10(ctr, key) == out[blk]).all(), (seed, ctr)
+
+
+def test_philox_every_counter_word_and_key_word_matters():
+    base = oracle.philox4x32_10([1, 2, 3, 4], [5, 6])
+    seen = {tuple(base)}
+    for i in range(4):
+        c = [1, 2, 3, 4]
+        c[i] ^= 0x80000000
+        seen.add(tuple(oracle.philox4x32_10(c, [5, 6])))
+    seen.add(tuple(oracle.philox4x32_10([1, 2, 3, 4], [5 ^ 1, 6])))
+    seen.add(tuple(oracle.philox4x32_10([1, 2, 3, 4], [5, 6 ^ 1])))
+    # swapping two counter words is a different counter
+    seen.add(tuple(oracle.philox4x32_10([1, 2, 4, 3], [5, 6])))
+    seen.add(tuple(oracle.philox4x32_10([2, 1, 3, 4], [5, 6])))
+    assert len(seen) == 9
+
+
+def test_uniform_counter_layout_and_mapping():
+    """u = ((r >> 9) + 0.5) / 2^23 of word `lane` of philox(((stream << 30) | j, b, pos, step), (seed lo, seed hi))."""
+    seed = 0xDEADBEEF12345678
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for stream, j, b, pos, step, lane in [(0, 0, 0, 0, 0, 0), (1, 31615, 63, 31, 1000, 3), (1, 5, 2, 7, 9, 1),
+                                          (0, 0, 17, 63, 0xFFFFFFFF, 0), (2, (1 << 30) - 1, 1, 1, 1, 2)]:
+        r = oracle.philox4x32_10([(stream << 30) | j, b, pos, step], key)
+        want = (float(r[lane] >> 9) + 0.5) / 8388608.0
+        got = oracle.uniform(seed, stream, j, b, pos, step, lane)
+        assert got == want
+        assert 0.0 < got < 1.0
+        assert float(np.float32(got)) == got  # exactly representable in binary32
+
+
+def test_uniforms_are_uniform():
+    us = np.array([oracle.uniform(42, 0, 0, b, b % 7, 3, 0) for b in range(40000)])
+    assert stats.kstest(us, "uniform").pvalue > 1e-3
+    us = np.array([oracle.uniform(42, 1, v >> 2, 5, 1, 3, v & 3) for v in range(40000)])
+    assert stats.kstest(us, "uniform").pvalue > 1e-3
+    assert abs(np.corrcoef(us[:-1], us[1:])[0, 1]) < 0.02
+
+
+# ----------------------------------------------------------------- softmax ----
+@pytest.mark.parametrize("T", [1.0, 0.7, 2.5])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_laws_match_library_softmax(T, dtype):
+    g = torch.Generator().manual_seed(3)
+    V = 777
+    p = (torch.randn(V, generator=g) * 3).to(dtype)
+    q = (torch.randn(V, generator=g) * 3 + 1.5).to(dtype)
+    pi, rho, resid, alpha = oracle.row_laws(p, q, T)
+    # T is handed over as a binary32 number, as in the library's C signature
+    T32 = float(np.float32(T))
+    want_pi = _softmax64(p.to(torch.float64).numpy(), T32)
+    want_rho = _softmax64(q.to(torch.float64).numpy(), T32)
+    np.testing.assert_allclose(pi, want_pi, rtol=1e-12, atol=0)
+    np.testing.assert_allclose(rho, want_rho, rtol=1e-12, atol=0)
+    assert abs(pi.sum() - 1) < 1e-12 and abs(rho.sum() - 1) < 1e-12
+    # adding a constant to a row changes nothing (softmax shift invariance); exact shift in fp32
+    if dtype == torch.float32:
+        pi2, _, _, _ = oracle.row_laws((p.double() + 4.0).float(), q, T)
+        np.testing.assert_allclose(pi2, want_pi, rtol=1e-6)
+
+
+def test_minus_inf_logit_is_probability_zero():
+    p = _f32([0.0, -np.inf, 1.0, -np.inf])
+    q = _f32([-np.inf, 0.0, 0.0, 0.0])
+    pi, rho, resid, alpha = oracle.row_laws(p, q, 1.0)
+    assert pi[1] == 0 and pi[3] == 0 and rho[0] == 0
+    np.testing.assert_allclose(pi, _softmax64([0.0, -np.inf, 1.0, -np.inf]), rtol=1e-14)
+
+
+# ---------------------------------------- acceptance probability (P1), residual (P3) ----
+def test_acceptance_probability_and_residual_identities():
+    rng = np.random.default_rng(0)
+    for V in (2, 4, 16, 300):
+        for T in (1.0, 0.6):
+            lp = rng.normal(0, 2, V).astype(np.float32)
+            lq = (lp + rng.normal(0, 1.0, V)).astype(np.float32)
+            pi, rho, resid, alpha = oracle.row_laws(_f32(lp), _f32(lq), T)
+            T32 = float(np.float32(T))
+            PI, RHO = _softmax64(lp, T32), _softmax64(lq, T32)
+            # P1: sum_x rho(x) min{1, pi(x)/rho(x)} = sum_z min{pi, rho}
+            acc = float(np.sum(RHO * np.minimum(1.0, PI / RHO)))
+            assert abs(alpha - acc) < 1e-12
+            assert abs(alpha - np.minimum(PI, RHO).sum()) < 1e-12
+            # P3: the residual is a probability law, zero wherever pi <= rho, proportional to pi - rho elsewhere
+            assert abs(resid.sum() - 1.0) < 1e-9
+            assert (resid[PI <= RHO] == 0).all()
+            pos = PI > RHO
+            np.testing.assert_allclose(resid[pos], (PI - RHO)[pos] / (1.0 - acc), rtol=1e-9)
+            # normaliser identity: sum [pi - rho]_+ = 1 - sum min
+            assert abs(np.maximum(PI - RHO, 0).sum() - (1 - alpha)) < 1e-12
+
+
+def test_emitted_token_law_equals_target_by_exact_enumeration_single_position():
+    """Pr(commit x) = rho(x) min{1, pi/rho}(x) + (1 - alpha) resid(x) must equal pi(x) (proof of Theorem 1)."""
+    rng = np.random.default_rng(1)
+    for _ in range(20):
+        V = 4
+        lp = rng.normal(0, 1.5, V).astype(np.float32)
+        lq = rng.normal(0, 1.5, V).astype(np.float32)
+        pi, rho, resid, alpha = oracle.row_laws(_f32(lp), _f32(lq), 1.0)
+        emitted = rho * np.minimum(1.0, pi / rho) + (1.0 - alpha) * resid
+        np.testing.assert_allclose(emitted, _softmax64(lp), rtol=1e-12)
+
+
+# --------------------------------------------------- the random procedure itself ----
+def _run(q, p, tok, T, seed, step, row_len=None):
+    r = oracle.spec_verify(q, p, tok, T, seed, step, row_len=row_len)
+    assert r["status"] == 0
+    return r
+
+
+def test_acceptance_frequency_matches_sum_min():
+    """Monte Carlo over Philox draws: accepted fraction within a binomial interval of alpha."""
+    rng = np.random.default_rng(2)
+    V, B = 4, 200000
+    lp = np.array([0.3, -0.8, 1.1, 0.0], np.float32)
+    lq = np.array([-0.2, 0.9, 0.1, 0.4], np.float32)
+    PI, RHO = _softmax64(lp), _softmax64(lq)
+    alpha = np.minimum(PI, RHO).sum()
+    tok = _draw_from(RHO, B, rng).reshape(B, 1)
+    r = _run(_tile(lq, B), _tile(lp, B), tok, 1.0, seed=11, step=5)
+    frac = (r["accept_len"] == 1).mean()
+    assert abs(frac - alpha) < 5 * np.sqrt(alpha * (1 - alpha) / B)
+    # per draft token the accepted fraction is min{1, pi/rho}
+    for x in range(V):
+        sel = tok[:, 0] == x
+        want = min(1.0, PI[x] / RHO[x])
+        got = (r["accept_len"][sel] == 1).mean()
+        assert abs(got - want) < 5 * np.sqrt(max(want * (1 - want), 1e-4) / sel.sum())
+
+
+@pytest.mark.parametrize("V", [4, 16])
+def test_residual_draw_frequencies_chi_square(V):
+    rng = np.random.default_rng(3 + V)
+    B = 300000
+    lp = rng.normal(0, 1.2, V).astype(np.float32)
+    lq = rng.normal(0, 1.2, V).astype(np.float32)
+    PI, RHO = _softmax64(lp), _softmax64(lq)
+    res = np.maximum(PI - RHO, 0)
+    res /= res.sum()
+    tok = _draw_from(RHO, B, rng).reshape(B, 1)
+    r = _run(_tile(lq, B), _tile(lp, B), tok, 1.0, seed=99, step=1)
+    rej = r["accept_len"] == 0
+    Z = r["tokens"][rej, 0]
+    assert rej.sum() > 10000
+    assert (res[Z] > 0).all()  # never a token outside the residual's support
+    support = np.nonzero(res > 0)[0]
+    counts = np.array([(Z == x).sum() for x in support])
+    chi = stats.chisquare(counts, res[support] * counts.sum())
+    assert chi.pvalue > 1e-4, chi
+    # confidence of the corrected token is the TARGET probability of it, not the residual's
+    np.testing.assert_allclose(r["conf"][rej, 0], PI[Z], rtol=1e-12)
+
+
+def test_single_position_emitted_token_law_chi_square():
+    rng = np.random.default_rng(5)
+    V, B = 4, 300000
+    lp = np.array([1.0, 0.2, -0.5, 0.4], np.float32)
+    lq = np.array([0.0, 0.8, 0.3, -1.0], np.float32)
+    PI, RHO = _softmax64(lp), _softmax64(lq)
+    tok = _draw_from(RHO, B, rng).reshape(B, 1)
+    r = _run(_tile(lq, B), _tile(lp, B), tok, 1.0, seed=2024, step=0)
+    counts = np.bincount(r["tokens"][:, 0], minlength=V)
+    assert stats.chisquare(counts, PI * B).pvalue > 1e-4
+
+
+def test_joint_law_of_a_window_V4_K2_exact_enumeration_and_chi_square():
+    """Theorem 1 at V = 4, K = 2 with a prefix-dependent target for position 2.
+
+    Exact part: from the oracle's per-position laws, Pr(x1, x2) enumerated over
+    drafts and over accept/reject outcomes equals pi1(x1) * pi2(x2 | x1).
+    Monte-Carlo part: running the procedure (round 1 over both positions, round 2
+    over position 2 for the windows that rejected at position 1) reproduces it."""
+    rng = np.random.default_rng(7)
+    V = 4
+    lp1 = rng.normal(0, 1, V).astype(np.float32)
+    lq1 = rng.normal(0, 1, V).astype(np.float32)
+    lp2 = rng.normal(0, 1, (V, V)).astype(np.float32)   # target logits of position 2 given token at position 1
+    lq2 = rng.normal(0, 1, V).astype(np.float32)        # the draft does not see the prefix
+    PI1, RHO1, RHO2 = _softmax64(lp1), _softmax64(lq1), _softmax64(lq2)
+    PI2 = _softmax64(lp2)
+    want = PI1[:, None] * PI2
+
+    # exact enumeration through the oracle's laws
+    pi1, rho1, res1, a1 = oracle.row_laws(_f32(lp1), _f32(lq1), 1.0)
+    emit1 = rho1 * np.minimum(1, pi1 / rho1) + (1 - a1) * res1
+    joint = np.zeros((V, V))
+    for x1 in range(V):
+        pi2, rho2, res2, a2 = oracle.row_laws(_f32(lp2[x1]), _f32(lq2), 1.0)
+        emit2 = rho2 * np.minimum(1, pi2 / rho2) + (1 - a2) * res2
+        joint[x1] = emit1[x1] * emit2
+    np.testing.assert_allclose(joint, want, rtol=1e-12)
+
+    # the procedure
+    B = 300000
+    d1 = _draw_from(RHO1, B, rng)
+    d2 = _draw_from(RHO2, B, rng)
+    q = np.stack([np.broadcast_to(lq1, (B, V)), np.broadcast_to(lq2, (B, V))], axis=1)
+    p = np.stack([np.broadcast_to(lp1, (B, V)), lp2[d1]], axis=1)  # verification input uses the DRAFT prefix
+    r = _run(_f32(q), _f32(p), np.stack([d1, d2], 1), 1.0, seed=5, step=0)
+    x1 = r["tokens"][:, 0].copy()
+    x2 = r["tokens"][:, 1].copy()
+    a = r["accept_len"]
+    assert ((a == 0) == (x2 == -1)).all()      # a rejection at position 1 discards the draft at position 2
+    redo = np.nonzero(a == 0)[0]
+    d2b = _draw_from(RHO2, len(redo), rng)
+    r2 = _run(_tile(lq2, len(redo)), _f32(lp2[x1[redo]][:, None, :]), d2b.reshape(-1, 1), 1.0, seed=5, step=1)
+    x2[redo] = r2["tokens"][:, 0]
+    counts = np.zeros((V, V))
+    np.add.at(counts, (x1, x2), 1)
+    assert stats.chisquare(counts.ravel(), (want * B).ravel()).pvalue > 1e-4
+
+
+def test_identical_laws_accept_everything():
+    g = torch.Generator().manual_seed(0)
+    B, K, V = 64, 8, 50
+    q = torch.randn(B, K, V, generator=g)
+    tok = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    for seed in range(5):
+        r = _run(q, q.clone(), tok, 0.8, seed=seed, step=seed)
+        assert (r["accept_len"] == K).all()
+        assert np.isinf(r["gumbel_gap"]).all()  # the residual is never sampled
+        assert (r["tokens"] == tok.numpy()).all()
+        np.testing.assert_allclose(r["conf"], np.take_along_axis(_softmax64(q.numpy(), float(np.float32(0.8))), tok.numpy()[..., None].astype(np.int64), -1)[..., 0], rtol=1e-12)
+
+
+def _golden_theorem2():
+    rows = []
+    with open(os.path.join(GOLDEN, "theorem2_expected_length.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                a, k, e = line.split()
+                rows.append((float(a), int(k), float(e)))
+    return rows
+
+
+@pytest.mark.parametrize("alpha,K,expected", _golden_theorem2())
+def test_mean_committed_length_matches_theorem_2(alpha, K, expected):
+    """Two-token vocabulary with pi = (x, 1-x), rho = (1-x, x), x = 1 - alpha/2, so that
+    sum min(pi, rho) = alpha at every position; committed = min(accept_len + 1, K)."""
+    rng = np.random.default_rng(int(alpha * 1000) + K)
+    B = 100000
+    x = 1.0 - alpha / 2.0
+    with np.errstate(divide="ignore"):
+        lp = np.log(np.array([x, 1 - x])).astype(np.float32)
+        lq = np.log(np.array([1 - x, x])).astype(np.float32)
+    RHO = np.array([1 - x, x])
+    tok = _draw_from(RHO, B * K, rng).reshape(B, K)
+    r = _run(_tile(np.broadcast_to(lq, (K, 2)), B, K), _tile(np.broadcast_to(lp, (K, 2)), B, K), tok, 1.0, seed=31337, step=K)
+    committed = np.minimum(r["accept_len"] + 1, K)
+    sd = committed.std() / np.sqrt(B)
+    assert abs(committed.mean() - expected) < 5 * sd + 1e-9
+    assert ((r["tokens"] >= 0).sum(1) == committed).all()
+
+
+def test_mean_committed_length_unequal_alphas():
+    """Generalisation used for arbitrary logits: E[C] = sum_l prod_{i<l} alpha_i."""
+    rng = np.random.default_rng(8)
+    B, K, V = 100000, 4, 8
+    lq = rng.normal(0, 1, (K, V)).astype(np.float32)
+    lp = (lq + rng.normal(0, 0.8, (K, V))).astype(np.float32)
+    PI, RHO = _softmax64(lp), _softmax64(lq)
+    alphas = np.minimum(PI, RHO).sum(1)
+    want = sum(np.prod(alphas[:l]) for l in range(K))
+    tok = np.stack([_draw_from(RHO[i], B, rng) for i in range(K)], 1)
+    r = _run(_tile(lq, B, K), _tile(lp, B, K), tok, 1.0, seed=77, step=3)
+    committed = np.minimum(r["accept_len"] + 1, K)
+    assert abs(committed.mean() - want) < 5 * committed.std() / np.sqrt(B)
+
+
+def test_first_rejection_stops_the_window_and_sentinels():
+    rng = np.random.default_rng(9)
+    B, K, V = 2000, 6, 12
+    lq = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    lp = (lq + rng.normal(0, 1.5, (B, K, V))).astype(np.float32)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    r = _run(_f32(lq), _f32(lp), tok, 1.0, seed=1, step=2)
+    PI, RHO = _softmax64(lp), _softmax64(lq)
+    for b in range(B):
+        a = r["accept_len"][b]
+        # replay the scan with the published uniforms
+        for i in range(K):
+            u = oracle.uniform(1, 0, 0, b, i, 2, 0)
+            ok = u <= min(1.0, PI[b, i, tok[b, i]] / RHO[b, i, tok[b, i]])
+            if not ok:
+                assert a == i
+                break
+        else:
+            assert a == K
+        assert (r["tokens"][b, :a] == tok[b, :a]).all()
+        assert (r["tokens"][b, a + 1:] == -1).all() and (r["conf"][b, a + 1:] == -1.0).all()
+        if a < K:
+            z = r["tokens"][b, a]
+            assert PI[b, a, z] > RHO[b, a, z]
+            assert abs(r["conf"][b, a] - PI[b, a, z]) < 1e-12
+
+
+def test_row_len_limits_the_window():
+    rng = np.random.default_rng(10)
+    B, K, V = 50, 5, 9
+    lq = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    row_len = rng.integers(0, K + 1, B).astype(np.int32)
+    r = _run(_f32(lq), _f32(lq), tok, 1.0, seed=1, step=2, row_len=row_len)
+    assert (r["accept_len"] == row_len).all()
+    for b in range(B):
+        assert (r["tokens"][b, row_len[b]:] == -1).all()
+
+
+def test_greedy_temperature_zero_is_argmax_compare():
+    rng = np.random.default_rng(12)
+    B, K, V = 300, 5, 40
+    lp = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    lp[:, :, 7] = lp[:, :, 3]  # exact ties: the lowest index wins
+    lq = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    top = lp.argmax(-1)  # numpy returns the first maximum
+    tok = np.where(rng.random((B, K)) < 0.7, top, rng.integers(0, V, (B, K))).astype(np.int32)
+    r = _run(_f32(lq), _f32(lp), tok, 0.0, seed=1, step=2)
+    PI1 = _softmax64(lp)
+    for b in range(B):
+        mism = np.nonzero(tok[b] != top[b])[0]
+        a = mism[0] if len(mism) else K
+        assert r["accept_len"][b] == a
+        assert (r["tokens"][b, :a] == tok[b, :a]).all()
+        if a < K:
+            assert r["tokens"][b, a] == top[b, a]
+        n = min(a + 1, K)
+        np.testing.assert_allclose(r["conf"][b, :n], PI1[b, np.arange(n), r["tokens"][b, :n]], rtol=1e-12)
+    assert np.isinf(r["gumbel_gap"]).all() and np.isinf(r["accept_margin"]).all()
+
+
+def test_zero_draft_probability_conventions():
+    # rho(x) = 0 < pi(x): accept.  pi(x) = rho(x) = 0: reject, and the replacement comes from the residual.
+    lp = _f32([[[0.0, 0.0, -np.inf]]])
+    lq = _f32([[[-np.inf, 0.0, -np.inf]]])
+    for step in range(20):
+        r = _run(lq, lp, np.array([[0]], np.int32), 1.0, 3, step)
+        assert r["accept_len"][0] == 1 and r["tokens"][0, 0] == 0 and r["conf"][0, 0] == 0.5
+        r = _run(lq, lp, np.array([[2]], np.int32), 1.0, 3, step)
+        assert r["accept_len"][0] == 0 and r["tokens"][0, 0] == 0  # residual = (0.5, 0, 0)/0.5
+    # forced rejection with zero residual mass (pi = rho) commits arg-max pi
+    lp = _f32([[[0.0, 1.0, -np.inf]]])
+    r = _run(lp, lp, np.array([[2]], np.int32), 1.0, 3, 0)
+    assert r["accept_len"][0] == 0 and r["tokens"][0, 0] == 1
+
+
+def test_data_errors_are_reported_per_window():
+    rng = np.random.default_rng(13)
+    B, K, V = 4, 3, 6
+    lq = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    lp = lq.copy()
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    bad = lp.copy()
+    bad[1, 2, 4] = np.nan
+    r = oracle.spec_verify(_f32(lq), _f32(bad), tok, 1.0, 0, 0)
+    assert r["status"] == oracle.ERR_NONFINITE and r["accept_len"][1] == -1 and (r["accept_len"][[0, 2, 3]] == K).all()
+    assert (r["tokens"][1] == -1).all()
+    bad = lp.copy()
+    bad[2, 0, :] = -np.inf
+    assert oracle.spec_verify(_f32(lq), _f32(bad), tok, 1.0, 0, 0)["status"] == oracle.ERR_NONFINITE
+    bad = lq.copy()
+    bad[0, 1, 1] = np.inf
+    assert oracle.spec_verify(_f32(bad), _f32(lp), tok, 1.0, 0, 0)["status"] == oracle.ERR_NONFINITE
+    t2 = tok.copy()
+    t2[3, 1] = V
+    r = oracle.spec_verify(_f32(lq), _f32(lp), t2, 1.0, 0, 0)
+    assert r["status"] == oracle.ERR_TOKEN_RANGE and r["accept_len"][3] == -1
+    # entries past row_len are never looked at
+    r = oracle.spec_verify(_f32(lq), _f32(lp), t2, 1.0, 0, 0, row_len=np.array([3, 3, 3, 1], np.int32))
+    assert r["status"] == 0 and r["accept_len"][3] == 1
+    assert oracle.spec_verify(_f32(lq), _f32(lp), tok, -1.0, 0, 0)["status"] == oracle.ERR_INVALID_ARG
+
+
+def test_stream_depends_on_seed_step_batch_and_position():
+    rng = np.random.default_rng(14)
+    B, K, V = 256, 4, 16
+    lq = rng.normal(0, 1, (1, K, V)).astype(np.float32)
+    lp = (lq + rng.normal(0, 1.5, (1, K, V))).astype(np.float32)
+    q, p = _tile(lq[0], B, K), _tile(lp[0], B, K)
+    tok = np.broadcast_to(rng.integers(0, V, (1, K)), (B, K)).astype(np.int32).copy()
+    base = _run(q, p, tok, 1.0, 1, 1)
+    assert len(set(base["accept_len"].tolist())) > 1            # batch rows draw different numbers
+    assert (_run(q, p, tok, 1.0, 1, 1)["tokens"] == base["tokens"]).all()  # replayable
+    assert (_run(q, p, tok, 1.0, 1, 2)["tokens"] != base["tokens"]).any()
+    assert (_run(q, p, tok, 1.0, 2, 1)["tokens"] != base["tokens"]).any()
+    assert (_run(q, p, tok, 1.0, 1 << 32 | 1, 1)["tokens"] != base["tokens"]).any()  # high seed word is used
+
+
+def test_bf16_logits_are_read_exactly():
+    g = torch.Generator().manual_seed(1)
+    B, K, V = 3, 4, 64
+    q = torch.randn(B, K, V, generator=g).to(torch.bfloat16)
+    p = (q.float() + 0.5 * torch.randn(B, K, V, generator=g)).to(torch.bfloat16)
+    tok = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    a = oracle.spec_verify(q, p, tok, 1.0, 4, 4)
+    b = oracle.spec_verify(q.float(), p.float(), tok, 1.0, 4, 4)
+    assert (a["tokens"] == b["tokens"]).all() and (a["conf"] == b["conf"]).all()
+
+
+def test_leading_dimension_padding_is_ignored():
+    rng = np.random.default_rng(15)
+    B, K, V, ld = 5, 3, 10, 16
+    lq = rng.normal(0, 1, (B, K, ld)).astype(np.float32)
+    lp = rng.normal(0, 1, (B, K, ld)).astype(np.float32)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    a = oracle.spec_verify(_f32(lq), _f32(lp), tok, 1.0, 4, 4, V=V)
+    lq2, lp2 = lq.copy(), lp.copy()
+    lq2[:, :, V:] = 50.0
+    lp2[:, :, V:] = np.nan
+    b = oracle.spec_verify(_f32(lq2), _f32(lp2), tok, 1.0, 4, 4, V=V)
+    c = oracle.spec_verify(_f32(lq[:, :, :V].copy()), _f32(lp[:, :, :V].copy()), tok, 1.0, 4, 4)
+    assert a["status"] == b["status"] == c["status"] == 0
+    assert (a["tokens"] == b["tokens"]).all() and (a["tokens"] == c["tokens"]).all()
+    assert (a["conf"] == c["conf"]).all()
+
+
+# ---------------------------------------------------------------- LowConf ----
+def test_remask_select_matches_library_stable_sort():
+    rng = np.random.default_rng(16)
+    for B, L, k in [(3, 17, 5), (8, 256, 8), (2, 1024, 2), (4, 33, 40), (1, 1, 1), (2, 9, 0)]:
+        conf = rng.random((B, L)).astype(np.float32)
+        conf[rng.random((B, L)) < 0.3] = np.float32(0.25)       # many exact ties
+        mask = (rng.random((B, L)) < 0.6).astype(np.uint8)
+        pos, cnt = oracle.remask_select(conf, mask, k)
+        for b in range(B):
+            cand = np.nonzero(mask[b])[0]
+            order = cand[np.argsort(conf[b, cand], kind="stable")]
+            n = min(k, len(cand))
+            assert cnt[b] == n
+            assert (pos[b, :n] == order[:n]).all() and (pos[b, n:] == -1).all()
+
+
+def test_remask_select_brute_force_all_tie_patterns():
+    L, k = 5, 3
+    levels = [np.float32(0.1), np.float32(0.5), np.float32(0.9)]
+    for pattern in itertools.product(range(3), repeat=L):
+        conf = np.array([[levels[i] for i in pattern]], np.float32)
+        for mbits in (0b11111, 0b10110, 0b00001, 0):
+            mask = np.array([[(mbits >> i) & 1 for i in range(L)]], np.uint8)
+            pos, cnt = oracle.remask_select(conf, mask, k)
+            cand = sorted((pattern[i], i) for i in range(L) if mask[0, i])
+            want = [i for _, i in cand][:k]
+            assert cnt[0] == len(want) and pos[0, :len(want)].tolist() == want

@@ -1,0 +1,131 @@
+/*
+ * fef.h - C ABI of the B200 (sm_100a) speculative-verification library for
+ * FeF-DLLM decoding.
+ *
+ * The library implements, on one GPU, the verification loop of the paper's
+ * full-sequence decoding algorithm (Algorithm 2, "for m = 1..b"; Section 3.2
+ * "Acceleration via Speculative Decoding"; the residual law defined before
+ * Algorithm 2) for B independent speculative windows at once, and the
+ * low-confidence selection LowConf_{n_rm} of the same algorithm.
+ *
+ * Conventions
+ *  - Pointers marked "device" must be device memory of the current CUDA device;
+ *    the caller owns every buffer.  The library allocates nothing, keeps no
+ *    state between calls and never synchronises: all work is enqueued on
+ *    `cuda_stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *  - The return value reports what the host can see (bad arguments, launch
+ *    failures).  Errors that only the data reveals are written to
+ *    `*device_status` by the kernels; nothing ever traps.
+ *  - No CPU fallback exists: without a CUDA device every compute entry point
+ *    returns FEF_ERR_CUDA.
+ */
+#ifndef FEF_H
+#define FEF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FEF_OK = 0,
+    FEF_ERR_INVALID_ARG = 1, /* null pointer, size out of range, temperature < 0 or NaN   */
+    FEF_ERR_DTYPE = 2,       /* dtype is neither FEF_F32 nor FEF_BF16                     */
+    FEF_ERR_ALIGNMENT = 3,   /* logit base pointers or row pitch not 16-byte multiples    */
+    FEF_ERR_WORKSPACE = 4,   /* workspace missing, misaligned (256 B) or too small        */
+    FEF_ERR_CUDA = 5,        /* CUDA runtime error (see cudaGetLastError), or no device   */
+    FEF_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out            */
+    FEF_ERR_NONFINITE = 7,   /* device: NaN or +inf logit, or a row that is all -inf      */
+    FEF_ERR_TOKEN_RANGE = 8  /* device: a draft token outside [0, V)                      */
+} fef_status;
+
+typedef enum { FEF_F32 = 0, FEF_BF16 = 1 } fef_dtype;
+
+/* Largest window and selection sizes accepted. */
+#define FEF_MAX_B 65535
+#define FEF_MAX_K 64
+#define FEF_MAX_REMASK_L 8192
+
+/* Human-readable name of a status value (static storage, never NULL). */
+const char* fef_status_string(fef_status s);
+
+/*
+ * Bytes of device scratch fef_spec_verify needs for these sizes on the current
+ * CUDA device (it depends on the device's SM count).  Returns 0 for invalid
+ * sizes or when no device is available.  The scratch must be 256-byte aligned;
+ * its contents need not be initialised and are meaningless afterwards.
+ */
+size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt);
+
+/*
+ * One verification call over B speculative windows of K positions
+ * (Algorithm 2, lines "for m = 1 to b" .. "break"; acceptance rule and
+ * correction of Section 3.2; residual law pi' = [pi - rho]_+ / (1 - sum min{pi, rho})).
+ *
+ * With pi_i = softmax(target_logits[b,i,:] / T) and rho_i = softmax(draft_logits[b,i,:] / T),
+ * for each window b, scanning i = 0, 1, ... < n_b (n_b = row_len[b], or K):
+ *   u_i ~ U(0,1);  the draft x_i = draft_tokens[b,i] is accepted iff
+ *   u_i <= min{1, pi_i(x_i) / rho_i(x_i)};  accepted: tokens[b,i] = x_i, conf[b,i] = pi_i(x_i).
+ *   At the first rejection a: Z ~ pi'_a, tokens[b,a] = Z, conf[b,a] = pi_a(Z), stop.
+ * accept_len[b] = a (or n_b when nothing was rejected).  Entries after the last
+ * committed position get tokens = -1 and conf = -1.
+ *
+ * Temperature 0 is greedy: a draft is accepted iff it equals arg-max of the
+ * target logits (lowest index on ties), the replacement is that arg-max, no
+ * random numbers are used, draft_logits is not read, and conf is the T = 1
+ * softmax probability of the committed token.
+ *
+ * Random numbers: Philox4x32-10 keyed by (seed low word, seed high word) with
+ * counter ((stream << 30) | j, b, i, step).  Acceptance: stream 0, j = 0,
+ * output word 0.  Residual draw: Gumbel-max over x with [pi - rho]_+ > 0 of
+ * ln r_x - ln(-ln u_x), u_x from stream 1, j = x >> 2, output word x & 3;
+ * lowest x on exact ties.  A word r maps to u = ((r >> 9) + 0.5) * 2^-23.
+ * `step` must differ between calls that share a seed, or they reuse draws.
+ *
+ * Arguments
+ *   draft_logits, target_logits  device, [B, K, ld] row-major, dtype `dt`; only the first
+ *                    V entries of a row are read.  Base addresses and ld * sizeof(element)
+ *                    must be multiples of 16 bytes.  -inf entries are legal (probability 0).
+ *   draft_tokens     device, [B, K] int32, each in [0, V) for i < n_b
+ *   row_len          device, [B] int32 in [0, K] (drafts actually present), or NULL = K everywhere
+ *   B, K, V, ld      1 <= B <= FEF_MAX_B, 1 <= K <= FEF_MAX_K, V >= 1 (a row of at most 2^30 bytes),
+ *                    ld >= V (elements)
+ *   temperature      > 0 sampling, == 0 greedy; negative or NaN is FEF_ERR_INVALID_ARG
+ *   accept_len       device out, [B] int32
+ *   tokens           device out, [B, K] int32
+ *   conf             device out, [B, K] float32
+ *   workspace        device scratch of at least fef_spec_verify_workspace_bytes(...) bytes
+ *   device_status    device out, [1] int32, or NULL.  Set to FEF_OK at the start of the call,
+ *                    then to the largest device-side error.  Windows with a data error get
+ *                    accept_len = -1 and no committed tokens; other windows are unaffected.
+ *   cuda_stream      stream to enqueue on
+ */
+fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
+                           const int32_t* draft_tokens, const int32_t* row_len,
+                           int B, int K, int V, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step,
+                           int32_t* accept_len, int32_t* tokens, float* conf,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* cuda_stream);
+
+/*
+ * LowConf_k of Algorithm 2 ("Select R = LowConf_{n_rm}(C)"): for every batch
+ * row the k candidate positions of lowest confidence.
+ *
+ *   conf       device, [B, L] float32 confidences
+ *   mask       device, [B, L] uint8; a position is a candidate iff mask != 0
+ *   B, L, k    B >= 1, 1 <= L <= FEF_MAX_REMASK_L, k >= 0
+ *   positions  device out, [B, k] int32: candidates ordered by (conf ascending, index
+ *              ascending), padded with -1 when fewer than k candidates exist
+ *   count      device out, [B] int32 = min(k, number of candidates)
+ * -0 and +0 compare equal; NaN sorts after every number.
+ */
+fef_status fef_remask_select(const float* conf, const uint8_t* mask, int B, int L, int k,
+                             int32_t* positions, int32_t* count, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FEF_H */

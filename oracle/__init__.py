@@ -58,7 +58,7 @@ def lib() -> ctypes.CDLL:
             L.fef_oracle_row_laws.argtypes = [vp, vp, i32, i32, f32, vp, vp, vp, vp]
             L.fef_oracle_row_laws.restype = i32
             L.fef_oracle_spec_verify.argtypes = [
-                vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp,
+                vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, u32, vp, vp, vp, vp, vp,
             ]
             L.fef_oracle_spec_verify.restype = i32
             L.fef_oracle_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp]
@@ -131,8 +131,10 @@ def row_laws(p_logits, q_logits, temperature=1.0):
     return pi, rho, res, float(alpha[0])
 
 
-def spec_verify(draft_logits, target_logits, draft_tokens, temperature, seed, step, row_len=None, V=None):
-    """Run one verification call.  Logits are [B, K, ld]; ``V`` defaults to ld.
+def spec_verify(draft_logits, target_logits, draft_tokens, temperature, seed, step, row_len=None, V=None,
+                batch_offset=0):
+    """Run one verification call.  Logits are [B, K, ld]; ``V`` defaults to ld;
+    window b uses the random numbers of batch row ``batch_offset + b``.
 
     Returns a dict: status, accept_len [B], tokens [B,K], conf [B,K] (float64),
     accept_margin [B,K], gumbel_gap [B].
@@ -150,7 +152,7 @@ def spec_verify(draft_logits, target_logits, draft_tokens, temperature, seed, st
     margin = np.zeros((B, K), dtype=np.float64)
     gap = np.zeros(B, dtype=np.float64)
     st = lib().fef_oracle_spec_verify(
-        _ptr(q), _ptr(p), _ptr(tok), _ptr(rl), B, K, V, ld, dt, temperature, seed, step,
+        _ptr(q), _ptr(p), _ptr(tok), _ptr(rl), B, K, V, ld, dt, temperature, seed, step, batch_offset,
         _ptr(accept_len), _ptr(tokens), _ptr(conf), _ptr(margin), _ptr(gap),
     )
     return dict(status=st, accept_len=accept_len, tokens=tokens, conf=conf, accept_margin=margin, gumbel_gap=gap)

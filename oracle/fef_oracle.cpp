@@ -294,7 +294,7 @@ int fef_oracle_row_laws(const void* p_logits, const void* q_logits, int V, int d
 int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
                            const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
                            int64_t ld, int dtype, float temperature, uint64_t seed, uint32_t step,
-                           int32_t* accept_len, int32_t* tokens, double* conf,
+                           uint32_t batch_offset, int32_t* accept_len, int32_t* tokens, double* conf,
                            double* accept_margin, double* gumbel_gap) {
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
         return FEFO_ERR_INVALID_ARG;
@@ -318,7 +318,7 @@ int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
         o.gumbel_gap = gumbel_gap ? gumbel_gap + b : nullptr;
         const int n = row_len ? row_len[b] : K;
         const int st = verify_one_window(q, p, draft_tokens + window, n, K, V, ld, dtype,
-                                         (double)temperature, seed, (uint32_t)b, step, o);
+                                         (double)temperature, seed, batch_offset + (uint32_t)b, step, o);
         worst = std::max(worst, st);
     }
     return worst;

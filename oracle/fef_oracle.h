@@ -66,8 +66,11 @@ int fef_oracle_row_laws(const void* p_logits, const void* q_logits, int V, int d
  *   draft_logits, target_logits : [B, K, ld] (ld >= V), dtype F32 or BF16
  *   draft_tokens                : [B, K]
  *   row_len                     : [B] number of valid drafts (0..K), or NULL = K
- *   temperature                 : > 0 sampling; == 0 greedy (see DESIGN notes in
+ *   temperature                 : > 0 sampling; == 0 greedy (see the notes at the top of
  *                                 the .cpp); < 0 invalid
+ *   batch_offset                : window b draws its random numbers as batch row
+ *                                 batch_offset + b, so a slice of a larger batch can be
+ *                                 checked on its own
  * Outputs (caller allocated):
  *   accept_len [B]    index of first rejected draft, or row_len if none; -1 on a data error
  *   tokens     [B, K] committed tokens (accepted drafts, then the corrected token); -1 beyond
@@ -80,6 +83,7 @@ int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
                            const int32_t* draft_tokens, const int32_t* row_len,
                            int B, int K, int V, int64_t ld, int dtype,
                            float temperature, uint64_t seed, uint32_t step,
+                           uint32_t batch_offset,
                            int32_t* accept_len, int32_t* tokens, double* conf,
                            double* accept_margin, double* gumbel_gap);
 

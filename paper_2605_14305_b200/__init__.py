@@ -1,1 +1,171 @@
-"""B200-native speculative verification for FeF-DLLM decoding (binding added with the CUDA library)."""
+"""B200-native speculative verification for FeF-DLLM decoding.
+
+Thin Python binding of the C ABI declared in ``include/fef.h``: the functions
+here have the C entry points' names and only marshal arguments (torch tensors
+supply device memory and the current stream); every step of the computation
+runs in the CUDA library ``libfef.so``.  There is no CPU fallback: calling a
+compute function without the built library or without a CUDA device raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import NamedTuple, Optional
+
+import torch
+
+from . import _build
+
+FEF_OK, FEF_ERR_INVALID_ARG, FEF_ERR_DTYPE, FEF_ERR_ALIGNMENT, FEF_ERR_WORKSPACE = 0, 1, 2, 3, 4
+FEF_ERR_CUDA, FEF_ERR_TIMEOUT, FEF_ERR_NONFINITE, FEF_ERR_TOKEN_RANGE = 5, 6, 7, 8
+FEF_F32, FEF_BF16 = 0, 1
+FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
+
+EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_remask_select")
+
+_lib = None
+
+
+class FefError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, fef_status_string(status), status))
+
+
+def load(build_if_missing: bool = False) -> ctypes.CDLL:
+    """Load ``libfef.so`` (built in-tree by ``_build.build()``).  Raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        _build.build()
+    if not os.path.exists(_build.LIB_PATH):
+        raise RuntimeError(
+            "CUDA library %s is missing: build it with `python -m paper_2605_14305_b200._build` "
+            "(there is no CPU fallback)" % _build.LIB_PATH
+        )
+    L = ctypes.CDLL(_build.LIB_PATH)
+    vp, i32, i64, u32, u64, f32, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint32,
+                                       ctypes.c_uint64, ctypes.c_float, ctypes.c_size_t)
+    L.fef_status_string.argtypes = [i32]
+    L.fef_status_string.restype = ctypes.c_char_p
+    L.fef_spec_verify_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.fef_spec_verify_workspace_bytes.restype = sz
+    L.fef_spec_verify.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, sz, vp, vp]
+    L.fef_spec_verify.restype = i32
+    L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+    L.fef_remask_select.restype = i32
+    _lib = L
+    return L
+
+
+def fef_status_string(status: int) -> str:
+    return load().fef_status_string(int(status)).decode()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return FEF_F32
+    if t.dtype == torch.bfloat16:
+        return FEF_BF16
+    raise FefError(FEF_ERR_DTYPE, "fef_spec_verify")
+
+
+def _require_cuda(*tensors):
+    if not torch.cuda.is_available():
+        raise RuntimeError("no CUDA device: this library has no CPU path")
+    for t in tensors:
+        if t is not None and t.device.type != "cuda":
+            raise ValueError("all tensors must live on a CUDA device")
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def fef_spec_verify_workspace_bytes(B: int, K: int, V: int, dtype) -> int:
+    code = dtype if isinstance(dtype, int) else (FEF_F32 if dtype == torch.float32 else FEF_BF16)
+    return int(load().fef_spec_verify_workspace_bytes(B, K, V, code))
+
+
+class VerifyResult(NamedTuple):
+    accept_len: torch.Tensor   # [B] int32
+    tokens: torch.Tensor       # [B, K] int32
+    conf: torch.Tensor         # [B, K] float32
+    device_status: torch.Tensor  # [1] int32 (read it after synchronising)
+
+
+def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                    temperature: float, seed: int, step: int, row_len: Optional[torch.Tensor] = None,
+                    V: Optional[int] = None, out: Optional[VerifyResult] = None,
+                    workspace: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+    """Enqueue one verification call (see ``fef_spec_verify`` in include/fef.h).
+
+    ``draft_logits`` / ``target_logits``: ``[B, K, ld]`` CUDA tensors, float32 or
+    bfloat16, contiguous; ``V`` (default ``ld``) entries of each row are used.
+    Asynchronous on the current (or given) stream; outputs are reused from
+    ``out`` and scratch from ``workspace`` when given.
+    """
+    _require_cuda(draft_logits, target_logits, draft_tokens, row_len)
+    if draft_logits.dim() != 3 or draft_logits.shape != target_logits.shape or draft_logits.dtype != target_logits.dtype:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify")
+    if not (draft_logits.is_contiguous() and target_logits.is_contiguous() and draft_tokens.is_contiguous()):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify")
+    if draft_tokens.dtype != torch.int32 or (row_len is not None and row_len.dtype != torch.int32):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify")
+    B, K, ld = draft_logits.shape
+    V = ld if V is None else int(V)
+    code = _dtype_code(draft_logits)
+    dev = draft_logits.device
+    with torch.cuda.device(dev):
+        if out is None:
+            out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.float32, device=dev),
+                               torch.empty(1, dtype=torch.int32, device=dev))
+        if workspace is None:
+            workspace = torch.empty(max(fef_spec_verify_workspace_bytes(B, K, V, code), 256),
+                                    dtype=torch.uint8, device=dev)
+        st = load().fef_spec_verify(
+            draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
+            None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
+            int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
+            out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
+            workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_spec_verify")
+    return out
+
+
+def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions: Optional[torch.Tensor] = None,
+                      count: Optional[torch.Tensor] = None, stream=None):
+    """Enqueue LowConf_k (see ``fef_remask_select`` in include/fef.h).
+
+    ``conf`` ``[B, L]`` float32, ``mask`` ``[B, L]`` uint8 (or bool) ->
+    ``(positions [B, k] int32 padded with -1, count [B] int32)``.
+    """
+    _require_cuda(conf, mask)
+    if mask.dtype == torch.bool:
+        mask = mask.view(torch.uint8)
+    if conf.dim() != 2 or conf.shape != mask.shape or conf.dtype != torch.float32 or mask.dtype != torch.uint8:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_remask_select")
+    if not (conf.is_contiguous() and mask.is_contiguous()):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_remask_select")
+    B, L = conf.shape
+    dev = conf.device
+    with torch.cuda.device(dev):
+        if positions is None:
+            positions = torch.empty((B, max(int(k), 0)), dtype=torch.int32, device=dev)
+        if count is None:
+            count = torch.empty(B, dtype=torch.int32, device=dev)
+        st = load().fef_remask_select(conf.data_ptr(), mask.data_ptr(), B, L, int(k),
+                                      positions.data_ptr() if positions.numel() else None,
+                                      count.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_remask_select")
+    return positions, count
+
+
+__all__ = ["load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
+           "fef_spec_verify", "fef_remask_select", "EXPORTS"]

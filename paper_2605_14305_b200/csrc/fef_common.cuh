@@ -1,0 +1,190 @@
+// Device helpers shared by the kernels of the verification library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fef.h"
+
+namespace fef {
+
+// ------------------------------------------------------------------ sizes ----
+constexpr int kConsumerWarps = 16;                      // warps that do arithmetic in the streaming kernel
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kVecPerThread = 4;                        // 16-byte vectors per thread per tile
+constexpr int kTileBytes = kConsumerWarps * 32 * 16 * kVecPerThread;  // 32 KiB
+constexpr int kStages = 5;                              // ring depth: 160 KiB in flight per SM
+constexpr int kSpinLimit = 1 << 22;                     // bound on every mbarrier wait loop
+
+constexpr float kNoReference = -3.0e38f;                // "no reference yet" for the running softmax
+constexpr float kRescaleAbove = 1.152921504606847e18f;  // 2^60: a vector sum above this re-references
+
+// One partial result of the streaming kernel: a warp's share of one row.
+//   ref    reference exponent (log2 domain) the sum is relative to
+//   sum    sum_v 2^(l_v * c - ref) over the warp's elements (NaN when the data is bad)
+//   best   largest logit seen (greedy mode only)
+//   index  vocabulary id of `best`, lowest on ties (greedy mode only)
+struct __align__(16) Partial {
+    float ref;
+    float sum;
+    float best;
+    int index;
+};
+
+// Per-window hand-over from the scan kernel to the residual kernel.
+struct __align__(16) ResidualTask {
+    int pos;            // rejected position a, or -1 when the window has no residual draw
+    unsigned arrivals;  // CTAs of the residual kernel that have finished this window
+    double kp;          // log2 normaliser of the target law at a: pi(x) = 2^(l_x * c - kp)
+    double kq;          // same for the draft law
+};
+
+struct __align__(8) Candidate {
+    float w;  // r_x / (-ln u_x) in binary32, <= 0 when empty
+    int x;
+};
+
+// ------------------------------------------------------------ small maths ----
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// 2^(l * c - ref) with c = c_hi + c_lo (c_lo > 0 so that l = -inf stays -inf).
+__device__ __forceinline__ float exp2_scaled(float l, float c_hi, float c_lo, float ref) {
+    return ex2_approx(fmaf(l, c_lo, fmaf(l, c_hi, -ref)));
+}
+
+// Philox4x32-10 (Salmon et al. 2011): returns the four output words.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key) {
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, ctr.x), lo0 = M0 * ctr.x;
+        const uint32_t hi1 = __umulhi(M1, ctr.z), lo1 = M1 * ctr.z;
+        ctr = make_uint4(hi1 ^ ctr.y ^ key.x, lo1, hi0 ^ ctr.w ^ key.y, lo0);
+        key.x += W0;
+        key.y += W1;
+    }
+    return ctr;
+}
+
+// 23 random bits centred in their bin: u in (0, 1), exact in binary32.
+__device__ __forceinline__ float uniform_from_word(uint32_t r) {
+    return (static_cast<float>(r >> 9) + 0.5f) * (1.0f / 8388608.0f);
+}
+
+constexpr uint32_t kStreamAccept = 0u;
+constexpr uint32_t kStreamResidual = 1u;
+
+// ------------------------------------------------------ loads and unpacking ----
+template <int DT>
+struct Elem;
+template <>
+struct Elem<FEF_F32> {
+    static constexpr int kBytes = 4;
+    static constexpr int kPerVec = 4;
+};
+template <>
+struct Elem<FEF_BF16> {
+    static constexpr int kBytes = 2;
+    static constexpr int kPerVec = 8;
+};
+
+template <int DT>
+__device__ __forceinline__ void unpack(const uint4& w, float (&l)[Elem<DT>::kPerVec]) {
+    if constexpr (DT == FEF_F32) {
+        l[0] = __uint_as_float(w.x);
+        l[1] = __uint_as_float(w.y);
+        l[2] = __uint_as_float(w.z);
+        l[3] = __uint_as_float(w.w);
+    } else {
+        // a bfloat16 is the upper half of a binary32
+        l[0] = __uint_as_float(w.x << 16);
+        l[1] = __uint_as_float(w.x & 0xFFFF0000u);
+        l[2] = __uint_as_float(w.y << 16);
+        l[3] = __uint_as_float(w.y & 0xFFFF0000u);
+        l[4] = __uint_as_float(w.z << 16);
+        l[5] = __uint_as_float(w.z & 0xFFFF0000u);
+        l[6] = __uint_as_float(w.w << 16);
+        l[7] = __uint_as_float(w.w & 0xFFFF0000u);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ float load_logit(const void* row, int64_t v) {
+    if constexpr (DT == FEF_F32) {
+        return __ldg(static_cast<const float*>(row) + v);
+    } else {
+        const uint32_t h = __ldg(static_cast<const unsigned short*>(row) + v);
+        return __uint_as_float(h << 16);
+    }
+}
+
+__device__ __forceinline__ uint4 ld_global_nc_v4(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// --------------------------------------------------- mbarrier and bulk copy ----
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (int spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63) == 63 && *abort_flag) return false;
+    }
+    return false;
+}
+// 1-D bulk copy global -> shared, completion counted in bytes on `bar`.
+// dst, src and bytes must be multiples of 16.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst)),
+        "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Ordered 64-bit key for "largest w, then lowest x".
+__device__ __forceinline__ bool better(float w, int x, float w2, int x2) {
+    return w > w2 || (w == w2 && x < x2);
+}
+
+}  // namespace fef

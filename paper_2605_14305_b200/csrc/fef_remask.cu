@@ -1,0 +1,96 @@
+// fef_remask_select: LowConf_k of the paper's Algorithm 2 - per batch row, the k
+// candidate positions of lowest confidence in (confidence, index) order.
+//
+// One CTA per batch row.  Every position becomes a 64-bit key
+// (order-preserving image of the confidence << 32 | index), non-candidates get
+// the largest key, and the keys are sorted in shared memory with a bitonic
+// network; the first min(k, candidates) keys are the answer.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fef.h"
+
+namespace fef {
+
+constexpr int kRemaskThreads = 512;
+
+// Monotone map from binary32 (numeric order, -0 == +0, NaN last) to uint32.
+__device__ __forceinline__ uint32_t order_key(float f) {
+    uint32_t bits = __float_as_uint(f);
+    if (f != f) return 0xFFFFFFFEu;
+    if (bits == 0x80000000u) bits = 0u;
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kRemaskThreads) remask_kernel(const float* __restrict__ conf,
+                                                               const uint8_t* __restrict__ mask, int L, int k,
+                                                               int n_sort, int32_t* __restrict__ positions,
+                                                               int32_t* __restrict__ count) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
+    const int b = blockIdx.x;
+    const float* c = conf + static_cast<int64_t>(b) * L;
+    const uint8_t* m = mask + static_cast<int64_t>(b) * L;
+
+    int mine = 0;
+    for (int i = threadIdx.x; i < n_sort; i += kRemaskThreads) {
+        uint64_t key = ~0ull;
+        if (i < L && m[i] != 0) {
+            key = (static_cast<uint64_t>(order_key(c[i])) << 32) | static_cast<uint32_t>(i);
+            ++mine;
+        }
+        keys[i] = key;
+    }
+    __shared__ int s_total;
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+    if (mine) atomicAdd(&s_total, mine);
+
+    for (int size = 2; size <= n_sort; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int t = threadIdx.x; t < (n_sort >> 1); t += kRemaskThreads) {
+                const int lo = ((t / stride) * stride << 1) + (t % stride);
+                const int hi = lo + stride;
+                const bool ascending = ((lo & size) == 0);
+                const uint64_t a = keys[lo], z = keys[hi];
+                if ((a > z) == ascending) {
+                    keys[lo] = z;
+                    keys[hi] = a;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    const int total = s_total;
+    const int n = total < k ? total : k;
+    for (int t = threadIdx.x; t < k; t += kRemaskThreads)
+        positions[static_cast<int64_t>(b) * k + t] = t < n ? static_cast<int32_t>(keys[t] & 0xFFFFFFFFu) : -1;
+    if (threadIdx.x == 0) count[b] = n;
+}
+
+static bool g_remask_attr_done[64];
+
+}  // namespace fef
+
+extern "C" fef_status fef_remask_select(const float* conf, const uint8_t* mask, int B, int L, int k,
+                                         int32_t* positions, int32_t* count, void* cuda_stream) {
+    using namespace fef;
+    if (!conf || !mask || !count || B < 1 || L < 1 || L > FEF_MAX_REMASK_L || k < 0) return FEF_ERR_INVALID_ARG;
+    if (k > 0 && !positions) return FEF_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FEF_ERR_CUDA;
+    int n_sort = 2;
+    while (n_sort < L) n_sort <<= 1;
+    const size_t smem = static_cast<size_t>(n_sort) * sizeof(uint64_t);
+    if (smem > 48 * 1024 && !g_remask_attr_done[dev]) {
+        if (cudaFuncSetAttribute(remask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 FEF_MAX_REMASK_L * static_cast<int>(sizeof(uint64_t))) != cudaSuccess)
+            return FEF_ERR_CUDA;
+        g_remask_attr_done[dev] = true;
+    }
+    remask_kernel<<<B, kRemaskThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(conf, mask, L, k, n_sort,
+                                                                                     positions, count);
+    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}

@@ -1,0 +1,897 @@
+// fef_spec_verify: the verification loop of the paper's Algorithm 2 for B windows at once.
+//
+// Three kernels, enqueued back to back on the caller's stream:
+//   stream_kernel    reads every target and draft row exactly once (bulk-async copies into a
+//                    shared-memory ring) and leaves, per row, partial sums of
+//                    2^(l_v * c - ref), c = log2(e) / T, from which pi(x) and rho(x) follow
+//                    for any x  (the two softmax laws of Section 3.2);
+//   scan_kernel      per window: finishes the normalisers in double precision, draws u_i,
+//                    applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)}, finds the first rejection,
+//                    writes accepted tokens and confidences c_i = pi_i(x_i);
+//   residual_kernel  only for windows that rejected: Gumbel-max draw from
+//                    [pi - rho]_+ over the rejected row, then c = pi(Z).
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "fef.h"
+#include "fef_common.cuh"
+
+namespace fef {
+
+// Work split of one call, computed on the host and passed by value to the kernels.
+struct Geometry {
+    int B, K, V;
+    int units_per_row;    // 2: target row and draft row; 1 in greedy mode (target only)
+    int tile_bytes;       // bytes of one tile of a row (multiple of 8 KiB, <= kTileBytes)
+    int vec_bytes;        // bytes of a row covered by whole 16-byte vectors
+    int vec_elems;        // the same in elements; elements beyond are the row's "tail"
+    int tiles_per_unit;   // tiles per row (0 when a row holds no whole vector)
+    int grid;             // CTAs of the streaming kernel
+    int max_slots;        // partial-result slots per unit (>= CTAs that can share one unit)
+    int residual_ctas;    // CTAs per rejected row in the residual kernel
+    int64_t num_units;
+    int64_t num_tiles;
+    int64_t ld_bytes;     // row pitch in bytes
+};
+
+// CTA of the streaming kernel that owns global tile g (CTA c owns [c*NT/G, (c+1)*NT/G)).
+__host__ __device__ __forceinline__ int owner_of_tile(int64_t g, const Geometry& G) {
+    return static_cast<int>(((g + 1) * G.grid - 1) / G.num_tiles);
+}
+
+struct VerifyParams {
+    Geometry geo;
+    const char* target;   // p logits
+    const char* draft;    // q logits
+    const int32_t* draft_tokens;
+    const int32_t* row_len;
+    float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0
+    uint64_t seed;
+    uint32_t step;
+    int32_t* accept_len;
+    int32_t* tokens;
+    float* conf;
+    Partial* partials;
+    ResidualTask* tasks;
+    Candidate* candidates;
+    int32_t* status;
+};
+
+__device__ __forceinline__ void report(int32_t* status, int code) {
+    if (status) atomicMax(status, code);
+}
+
+// ============================================================ streaming ====
+// Running state of one thread for one row: sum of 2^(l*c - ref) and, in greedy
+// mode, the largest logit with its lowest index.
+struct RowState {
+    float ref, sum, best;
+    int index;
+    __device__ __forceinline__ void reset() {
+        ref = kNoReference;
+        sum = 0.f;
+        best = -INFINITY;
+        index = 0x7FFFFFFF;
+    }
+};
+
+template <int DT, bool GREEDY>
+__device__ __forceinline__ void absorb_vector(const uint4& w, int first_index, float c_hi, float c_lo,
+                                              RowState& st) {
+    constexpr int N = Elem<DT>::kPerVec;
+    float l[N], e[N];
+    unpack<DT>(w, l);
+#pragma unroll
+    for (int i = 0; i < N; ++i) e[i] = exp2_scaled(l[i], c_hi, c_lo, st.ref);
+    float vs;
+    if constexpr (N == 8)
+        vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    else
+        vs = (e[0] + e[1]) + (e[2] + e[3]);
+
+    if (!(vs <= kRescaleAbove)) {
+        // Rare: the reference is missing or far too low (or the data is bad).
+        // Move the reference to this vector's maximum and redo the vector.
+        float vmax = l[0];
+        bool bad = (l[0] != l[0]);
+#pragma unroll
+        for (int i = 1; i < N; ++i) {
+            vmax = fmaxf(vmax, l[i]);
+            bad = bad || (l[i] != l[i]);
+        }
+        if (bad || vmax == INFINITY) {
+            st.sum = __int_as_float(0x7FC00000);  // NaN marks the row as unusable
+        } else {
+            const float nref = fmaf(vmax, c_lo, vmax * c_hi);
+            st.sum *= ex2_approx(st.ref - nref);
+            st.ref = nref;
+#pragma unroll
+            for (int i = 0; i < N; ++i) e[i] = exp2_scaled(l[i], c_hi, c_lo, nref);
+            if constexpr (N == 8)
+                vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+            else
+                vs = (e[0] + e[1]) + (e[2] + e[3]);
+            st.sum += vs;
+        }
+    } else {
+        st.sum += vs;
+    }
+
+    if constexpr (GREEDY) {
+        float vmax = l[0];
+#pragma unroll
+        for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, l[i]);
+        if (vmax > st.best) {  // strict: an earlier (lower) index keeps a tie
+            int at = N - 1;
+#pragma unroll
+            for (int i = N - 2; i >= 0; --i)
+                if (l[i] == vmax) at = i;
+            st.best = vmax;
+            st.index = first_index + at;
+        }
+    }
+}
+
+template <bool GREEDY>
+__device__ __forceinline__ void flush_row(const RowState& st, int lane, Partial* out) {
+    float M = st.ref;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
+    float s = st.sum * ex2_approx(st.ref - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    float best = st.best;
+    int index = st.index;
+    if constexpr (GREEDY) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, index, o);
+            if (better(ob, oi, best, index)) {
+                best = ob;
+                index = oi;
+            }
+        }
+    }
+    if (lane == 0) {
+        Partial p;
+        p.ref = M;
+        p.sum = s;
+        p.best = best;
+        p.index = index;
+        *out = p;
+    }
+}
+
+// Position of a unit (a row of one of the two logit tensors) and whether it is in use.
+struct UnitInfo {
+    const char* base;  // first byte of the row
+    bool active;       // position < row_len of its window
+};
+__device__ __forceinline__ UnitInfo locate_unit(int64_t u, const VerifyParams& P) {
+    const Geometry& G = P.geo;
+    const int64_t row = (G.units_per_row == 2) ? (u >> 1) : u;
+    const bool is_draft = (G.units_per_row == 2) && (u & 1);
+    const int b = static_cast<int>(row / G.K);
+    const int i = static_cast<int>(row - static_cast<int64_t>(b) * G.K);
+    const int n = P.row_len ? __ldg(P.row_len + b) : G.K;
+    UnitInfo info;
+    info.base = (is_draft ? P.draft : P.target) + row * G.ld_bytes;
+    info.active = i < n;
+    return info;
+}
+
+template <int DT, bool GREEDY>
+__global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyParams P) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kTileBytes);
+    uint64_t* empty = full + kStages;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + kStages);
+
+    const Geometry& G = P.geo;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, kConsumerWarps);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    const int64_t g_begin = static_cast<int64_t>(blockIdx.x) * G.num_tiles / G.grid;
+    const int64_t g_end = (static_cast<int64_t>(blockIdx.x) + 1) * G.num_tiles / G.grid;
+    int64_t u = g_begin / G.tiles_per_unit;
+    int t = static_cast<int>(g_begin - u * G.tiles_per_unit);
+    int issued = 0;  // tiles put in flight (producer) / taken (consumers); identical sequences
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------ producer (one thread)
+        if (lane == 0) {
+            UnitInfo info = locate_unit(u, P);
+            for (int64_t g = g_begin; g < g_end; ++g) {
+                if (info.active) {
+                    const int s = issued % kStages;
+                    const uint32_t phase = (issued / kStages) & 1;
+                    if (!mbar_wait_bounded(empty + s, phase ^ 1u, abort_flag)) {
+                        *abort_flag = 1;
+                        report(P.status, FEF_ERR_TIMEOUT);
+                        break;
+                    }
+                    const int offset = t * G.tile_bytes;
+                    const int len = min(G.tile_bytes, G.vec_bytes - offset);
+                    mbar_arrive_expect_tx(full + s, static_cast<uint32_t>(len));
+                    bulk_copy_g2s(smem + s * kTileBytes, info.base + offset, static_cast<uint32_t>(len), full + s);
+                    ++issued;
+                }
+                if (++t == G.tiles_per_unit) {
+                    t = 0;
+                    ++u;
+                    if (g + 1 < g_end) info = locate_unit(u, P);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ consumers
+        RowState st;
+        st.reset();
+        bool have_row = false;
+        UnitInfo info = locate_unit(u, P);
+        for (int64_t g = g_begin; g < g_end; ++g) {
+            if (info.active) {
+                have_row = true;
+                const int s = issued % kStages;
+                const uint32_t phase = (issued / kStages) & 1;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(full + s, phase, abort_flag))) {
+                    *abort_flag = 1;
+                    report(P.status, FEF_ERR_TIMEOUT);
+                    break;
+                }
+                const int offset = t * G.tile_bytes;
+                const int len = min(G.tile_bytes, G.vec_bytes - offset);
+                const unsigned char* stage = smem + s * kTileBytes;
+                uint4 w[kVecPerThread];
+                int at[kVecPerThread];
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    at[j] = ((j * kConsumerWarps + warp) * 32 + lane) * 16;
+                    if (at[j] < len) w[j] = *reinterpret_cast<const uint4*>(stage + at[j]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
+                ++issued;
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j)
+                    if (at[j] < len)
+                        absorb_vector<DT, GREEDY>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+            }
+            if (++t == G.tiles_per_unit || g + 1 == g_end) {
+                if (have_row) {
+                    const int slot = static_cast<int>(blockIdx.x) - owner_of_tile(u * G.tiles_per_unit, G);
+                    flush_row<GREEDY>(st, lane, P.partials + (u * G.max_slots + slot) * kConsumerWarps + warp);
+                }
+                st.reset();
+                have_row = false;
+                if (t == G.tiles_per_unit) {
+                    t = 0;
+                    ++u;
+                    if (g + 1 < g_end) info = locate_unit(u, P);
+                }
+            }
+        }
+    }
+
+    __syncthreads();
+    // After an abort copies may still be in flight into this CTA's shared memory:
+    // give each a bounded chance to land before the CTA retires.
+    if (*abort_flag && warp == kConsumerWarps && lane == 0) {
+        const int first = issued > kStages ? issued - kStages : 0;
+        for (int k = first; k < issued; ++k) {
+            const int s = k % kStages;
+            const uint32_t phase = (k / kStages) & 1;
+            for (int spin = 0; spin < kSpinLimit; ++spin)
+                if (mbar_try_wait(full + s, phase)) break;
+        }
+    }
+}
+
+// ================================================================= scan ====
+struct RowNorm {
+    double M;     // reference exponent (log2 domain)
+    double S;     // sum_v 2^(l_v c - M)
+    float best;   // greedy: largest logit
+    int index;    // greedy: its lowest index
+    bool bad;
+};
+
+__device__ __forceinline__ double warp_max(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Combine the streaming kernel's partials of unit u (and the row's tail elements,
+// which the streaming kernel does not touch) into the row's normaliser.  Whole warp.
+template <int DT, bool GREEDY>
+__device__ RowNorm finish_row(int64_t u, const char* row, double c, const VerifyParams& P, int lane) {
+    const Geometry& G = P.geo;
+    int nrec = 0;
+    if (G.tiles_per_unit > 0) {
+        const int c_first = owner_of_tile(u * G.tiles_per_unit, G);
+        const int c_last = owner_of_tile((u + 1) * G.tiles_per_unit - 1, G);
+        nrec = (c_last - c_first + 1) * kConsumerWarps;
+    }
+    const Partial* rec = P.partials + u * G.max_slots * kConsumerWarps;
+    const int ntail = G.V - G.vec_elems;
+
+    double M = -INFINITY;
+    int bad = 0;
+    float best = -INFINITY;
+    int index = 0x7FFFFFFF;
+    for (int r = lane; r < nrec; r += 32) {
+        const Partial p = rec[r];
+        if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = 1;
+        if (p.sum > 0.f) M = fmax(M, static_cast<double>(p.ref));
+        if (GREEDY && better(p.best, p.index, best, index)) {
+            best = p.best;
+            index = p.index;
+        }
+    }
+    for (int j = lane; j < ntail; j += 32) {
+        const float l = load_logit<DT>(row, G.vec_elems + j);
+        if (l != l || l == INFINITY) bad = 1;
+        else if (l > -INFINITY) M = fmax(M, static_cast<double>(l) * c);
+        if (GREEDY && better(l, G.vec_elems + j, best, index)) {
+            best = l;
+            index = G.vec_elems + j;
+        }
+    }
+    M = warp_max(M);
+    bad = __any_sync(0xFFFFFFFFu, bad);
+    if (GREEDY) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, index, o);
+            if (better(ob, oi, best, index)) {
+                best = ob;
+                index = oi;
+            }
+        }
+    }
+
+    double S = 0.0;
+    if (!bad) {
+        for (int r = lane; r < nrec; r += 32) {
+            const Partial p = rec[r];
+            if (p.sum > 0.f) S += static_cast<double>(p.sum) * exp2(static_cast<double>(p.ref) - M);
+        }
+        for (int j = lane; j < ntail; j += 32) {
+            const float l = load_logit<DT>(row, G.vec_elems + j);
+            if (l > -INFINITY) S += exp2(static_cast<double>(l) * c - M);
+        }
+        S = warp_sum(S);
+    }
+    RowNorm out;
+    out.M = M;
+    out.S = S;
+    out.best = best;
+    out.index = index;
+    out.bad = bad || !(S > 0.0) || !(S < INFINITY);
+    return out;
+}
+
+constexpr int kScanWarps = 8;
+
+template <int DT, bool GREEDY>
+__global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const VerifyParams P) {
+    const Geometry& G = P.geo;
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+
+    __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
+    __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
+    __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
+
+    for (int i = warp; i < n; i += kScanWarps) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + i;
+        const char* prow = P.target + row * G.ld_bytes;
+        const char* qrow = P.draft + row * G.ld_bytes;
+        const RowNorm np = finish_row<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P, lane);
+        RowNorm nq;
+        nq.bad = false;
+        if constexpr (!GREEDY) nq = finish_row<DT, false>(2 * row + 1, qrow, c, P, lane);
+        if (lane == 0) {
+            const int x = __ldg(P.draft_tokens + row);
+            int err = 0, accept = 0, alt = -1;
+            float conf = -1.f, conf_alt = -1.f;
+            double kp = 0.0, kq = 0.0;
+            if (x < 0 || x >= G.V) {
+                err = FEF_ERR_TOKEN_RANGE;
+            } else if (np.bad || nq.bad) {
+                err = FEF_ERR_NONFINITE;
+            } else {
+                kp = np.M + log2(np.S);
+                const double lpx = load_logit<DT>(prow, x);
+                const double l2pi = lpx * c - kp;  // log2 pi(x)
+                conf = static_cast<float>(exp2(l2pi));
+                if constexpr (GREEDY) {
+                    accept = (x == np.index);
+                    alt = np.index;
+                    conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
+                } else {
+                    kq = nq.M + log2(nq.S);
+                    const double lqx = load_logit<DT>(qrow, x);
+                    if (lqx == -INFINITY) {
+                        accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
+                    } else {
+                        const double ratio = exp2(l2pi - (lqx * c - kq));
+                        const uint4 r = philox4x32_10(
+                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), P.step),
+                            make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+                        const double uacc = uniform_from_word(r.x);
+                        accept = uacc <= fmin(1.0, ratio);
+                    }
+                }
+            }
+            s_err[i] = err;
+            s_accept[i] = accept;
+            s_conf[i] = conf;
+            s_conf_alt[i] = conf_alt;
+            s_alt[i] = alt;
+            s_kp[i] = kp;
+            s_kq[i] = kq;
+        }
+    }
+    __syncthreads();
+
+    int err = 0, a = n;
+    for (int i = 0; i < n; ++i) err = max(err, s_err[i]);
+    for (int i = n - 1; i >= 0; --i)
+        if (!s_accept[i]) a = i;
+
+    const int i = threadIdx.x;
+    if (i < G.K) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + i;
+        int tok = -1;
+        float cf = -1.f;
+        if (!err) {
+            if (i < a) {
+                tok = __ldg(P.draft_tokens + row);
+                cf = s_conf[i];
+            } else if (GREEDY && i == a && a < n) {
+                tok = s_alt[i];
+                cf = s_conf_alt[i];
+            }
+        }
+        P.tokens[row] = tok;
+        P.conf[row] = cf;
+    }
+    if (threadIdx.x == 0) {
+        P.accept_len[b] = err ? -1 : a;
+        if (err) report(P.status, err);
+        ResidualTask task;
+        task.pos = (!GREEDY && !err && a < n) ? a : -1;
+        task.arrivals = 0u;
+        task.kp = task.pos >= 0 ? s_kp[a] : 0.0;
+        task.kq = task.pos >= 0 ? s_kq[a] : 0.0;
+        P.tasks[b] = task;
+    }
+}
+
+// ============================================================= residual ====
+constexpr int kResidualThreads = 256;
+constexpr int kMaxResidualCtas = kResidualThreads / 2;  // the last CTA looks at 2 candidates per CTA
+
+// -ln(u) for u = ((word >> 9) + 0.5) * 2^-23, accurate also when u is close to 1.
+__device__ __forceinline__ float neg_log_uniform(uint32_t word) {
+    const float k = static_cast<float>(word >> 9);
+    const float u = (k + 0.5f) * (1.0f / 8388608.0f);
+    const float t = (8388607.5f - k) * (1.0f / 8388608.0f);  // 1 - u, exact
+    const float series = t * fmaf(t, fmaf(t, fmaf(t, 0.25f, 1.0f / 3.0f), 0.5f), 1.0f);
+    const float direct = -0.6931471805599453f * lg2_approx(u);
+    return t < 0.015625f ? series : direct;
+}
+
+struct Top2 {
+    float w1, w2;
+    int x1, x2;
+    __device__ __forceinline__ void clear() {
+        w1 = w2 = 0.f;
+        x1 = x2 = 0x7FFFFFFF;
+    }
+    __device__ __forceinline__ void offer(float w, int x) {
+        if (better(w, x, w1, x1)) {
+            w2 = w1;
+            x2 = x1;
+            w1 = w;
+            x1 = x;
+        } else if (better(w, x, w2, x2)) {
+            w2 = w;
+            x2 = x;
+        }
+    }
+};
+
+// Exact (double) Gumbel score ln r_x - ln(-ln u_x) of vocabulary id x; -inf when r_x <= 0.
+template <int DT>
+__device__ double exact_score(int x, const char* prow, const char* qrow, double c, double kp, double kq,
+                              uint32_t b, uint32_t pos, const VerifyParams& P) {
+    const double lp = load_logit<DT>(prow, x);
+    const double lq = load_logit<DT>(qrow, x);
+    const double pi = exp2(lp * c - kp);
+    const double rho = exp2(lq * c - kq);
+    const double r = pi - rho;
+    if (!(r > 0.0)) return -INFINITY;
+    const uint4 w = philox4x32_10(
+        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, P.step),
+        make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+    const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
+    const double u = uniform_from_word(word);
+    return log(r) - log(-log(u));
+}
+
+// Block-wide arg-max of (score, lowest x).  Every thread gets the result.
+__device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double os = __shfl_xor_sync(0xFFFFFFFFu, score, o);
+        const int ox = __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        if (os > score || (os == score && ox < x)) {
+            score = os;
+            x = ox;
+        }
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) {
+        s_score[warp] = score;
+        s_x[warp] = x;
+    }
+    __syncthreads();
+    score = s_score[0];
+    x = s_x[0];
+    for (int w = 1; w < kResidualThreads / 32; ++w)
+        if (s_score[w] > score || (s_score[w] == score && s_x[w] < x)) {
+            score = s_score[w];
+            x = s_x[w];
+        }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kResidualThreads) residual_kernel(const VerifyParams P) {
+    constexpr int N = Elem<DT>::kPerVec;
+    const Geometry& G = P.geo;
+    const int b = blockIdx.y, part = blockIdx.x, parts = gridDim.x;
+    const ResidualTask task = P.tasks[b];
+    if (task.pos < 0) return;  // uniform over the CTA
+
+    const int64_t row = static_cast<int64_t>(b) * G.K + task.pos;
+    const char* prow = P.target + row * G.ld_bytes;
+    const char* qrow = P.draft + row * G.ld_bytes;
+    const float kp = static_cast<float>(task.kp), kq = static_cast<float>(task.kq);
+    const uint2 key = make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32));
+    const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(task.pos);
+
+    Top2 top;
+    top.clear();
+
+    // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x)
+    const int nvec = G.vec_elems / N;
+    const int v_begin = static_cast<int>(static_cast<int64_t>(part) * nvec / parts);
+    const int v_end = static_cast<int>(static_cast<int64_t>(part + 1) * nvec / parts);
+    for (int vec = v_begin + threadIdx.x; vec < v_end; vec += kResidualThreads) {
+        float lp[N], lq[N], r[N];
+        unpack<DT>(ld_global_nc_v4(prow + static_cast<int64_t>(vec) * 16), lp);
+        unpack<DT>(ld_global_nc_v4(qrow + static_cast<int64_t>(vec) * 16), lq);
+#pragma unroll
+        for (int i = 0; i < N; ++i)
+            r[i] = exp2_scaled(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled(lq[i], P.c_hi, P.c_lo, kq);
+#pragma unroll
+        for (int g4 = 0; g4 < N / 4; ++g4) {
+            const float rmax = fmaxf(fmaxf(r[4 * g4], r[4 * g4 + 1]), fmaxf(r[4 * g4 + 2], r[4 * g4 + 3]));
+            if (rmax > 0.f) {
+                const int x0 = vec * N + 4 * g4;
+                const uint4 w = philox4x32_10(
+                    make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
+                const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float ri = r[4 * g4 + i];
+                    if (ri > 0.f) top.offer(__fdividef(ri, neg_log_uniform(words[i])), x0 + i);
+                }
+            }
+        }
+    }
+    // tail elements (beyond the last whole vector) belong to part 0
+    if (part == 0) {
+        for (int x = G.vec_elems + threadIdx.x; x < G.V; x += kResidualThreads) {
+            const float lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
+            const float r = exp2_scaled(lp, P.c_hi, P.c_lo, kp) - exp2_scaled(lq, P.c_hi, P.c_lo, kq);
+            if (r > 0.f) {
+                const uint4 w = philox4x32_10(
+                    make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), ub, upos, P.step), key);
+                const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
+                top.offer(__fdividef(r, neg_log_uniform(word)), x);
+            }
+        }
+    }
+
+    // ---- CTA-wide best two
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ow1 = __shfl_xor_sync(0xFFFFFFFFu, top.w1, o), ow2 = __shfl_xor_sync(0xFFFFFFFFu, top.w2, o);
+        const int ox1 = __shfl_xor_sync(0xFFFFFFFFu, top.x1, o), ox2 = __shfl_xor_sync(0xFFFFFFFFu, top.x2, o);
+        top.offer(ow1, ox1);
+        top.offer(ow2, ox2);
+    }
+    __shared__ Top2 s_top[kResidualThreads / 32];
+    __shared__ int s_last;
+    __shared__ double s_score[kResidualThreads / 32];
+    __shared__ int s_x[kResidualThreads / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) s_top[warp] = top;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Top2 all = s_top[0];
+        for (int w = 1; w < kResidualThreads / 32; ++w) {
+            all.offer(s_top[w].w1, s_top[w].x1);
+            all.offer(s_top[w].w2, s_top[w].x2);
+        }
+        Candidate* out = P.candidates + (static_cast<int64_t>(b) * parts + part) * 2;
+        out[0].w = all.w1;
+        out[0].x = all.x1;
+        out[1].w = all.w2;
+        out[1].x = all.x2;
+        __threadfence();
+        const unsigned before = atomicAdd(&P.tasks[b].arrivals, 1u);
+        s_last = (before == static_cast<unsigned>(parts) - 1u);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    // ---- the last CTA of the window decides, in double precision, among the
+    //      candidates whose binary32 weight is within 2^-9 of the best one
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    const volatile Candidate* cand = P.candidates + static_cast<int64_t>(b) * parts * 2;
+    float w = 0.f;
+    int x = 0x7FFFFFFF;
+    if (static_cast<int>(threadIdx.x) < 2 * parts) {
+        w = cand[threadIdx.x].w;
+        x = cand[threadIdx.x].x;
+    }
+    double wbest = w;
+    int dummy = 0;
+    block_argmax(wbest, dummy, s_score, s_x);
+    double score = -INFINITY;
+    int Z = 0x7FFFFFFF;
+    if (w > 0.f && static_cast<double>(w) >= wbest * (1.0 - 1.0 / 512.0)) {
+        score = exact_score<DT>(x, prow, qrow, c, task.kp, task.kq, ub, upos, P);
+        if (score > -INFINITY) Z = x;
+    }
+    block_argmax(score, Z, s_score, s_x);
+
+    if (!(score > -INFINITY)) {
+        // Nothing survived in binary32 (the residual mass is at rounding level or zero):
+        // go over the whole row in double precision.
+        score = -INFINITY;
+        Z = 0x7FFFFFFF;
+        for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
+            const double s = exact_score<DT>(xx, prow, qrow, c, task.kp, task.kq, ub, upos, P);
+            if (s > score) {  // increasing xx: the lowest index keeps a tie
+                score = s;
+                Z = xx;
+            }
+        }
+        block_argmax(score, Z, s_score, s_x);
+        if (!(score > -INFINITY)) {
+            // [pi - rho]_+ is identically zero: commit arg-max of pi (= arg-max of the target logits)
+            score = -INFINITY;
+            Z = 0x7FFFFFFF;
+            for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
+                const double l = load_logit<DT>(prow, xx);
+                if (l > score) {
+                    score = l;
+                    Z = xx;
+                }
+            }
+            block_argmax(score, Z, s_score, s_x);
+        }
+    }
+    if (threadIdx.x == 0) {
+        const double lp = load_logit<DT>(prow, Z);
+        P.tokens[row] = Z;
+        P.conf[row] = static_cast<float>(exp2(lp * c - task.kp));
+    }
+}
+
+// ================================================================= host ====
+static int g_sm_count[64];
+static bool g_attr_done[64][4];
+
+static int sm_count_of_current_device(int* device_out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (g_sm_count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        g_sm_count[dev] = n;
+    }
+    if (device_out) *device_out = dev;
+    return g_sm_count[dev];
+}
+
+static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool greedy, int sm_count, Geometry* out) {
+    if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V || sm_count < 1) return false;
+    if (dt != FEF_F32 && dt != FEF_BF16) return false;
+    const int esize = dt == FEF_F32 ? 4 : 2;
+    if (static_cast<int64_t>(V) * esize > (1ll << 30)) return false;
+    Geometry G;
+    G.B = B;
+    G.K = K;
+    G.V = V;
+    G.units_per_row = greedy ? 1 : 2;
+    G.ld_bytes = ld * esize;
+    G.vec_bytes = static_cast<int>((static_cast<int64_t>(V) * esize) / 16 * 16);
+    G.vec_elems = G.vec_bytes / esize;
+    G.num_units = static_cast<int64_t>(B) * K * G.units_per_row;
+    const int64_t cta_target = sm_count;
+    // the largest tile that still leaves every CTA several tiles to pipeline
+    G.tile_bytes = kTileBytes;
+    while (G.tile_bytes > 8192 &&
+           G.num_units * ((G.vec_bytes + G.tile_bytes - 1) / G.tile_bytes) < 8 * cta_target)
+        G.tile_bytes >>= 1;
+    G.tiles_per_unit = (G.vec_bytes + G.tile_bytes - 1) / G.tile_bytes;
+    G.num_tiles = G.num_units * G.tiles_per_unit;
+    G.grid = static_cast<int>(G.num_tiles < cta_target ? G.num_tiles : cta_target);
+    if (G.grid < 1) G.grid = 1;
+    const int64_t min_tiles_per_cta = G.num_tiles > 0 ? G.num_tiles / G.grid : 1;
+    G.max_slots = G.tiles_per_unit > 0 ? static_cast<int>((G.tiles_per_unit - 1) / min_tiles_per_cta) + 2 : 1;
+    int parts = (2 * sm_count + B - 1) / B;
+    const int nvec = G.vec_bytes / 16;
+    const int max_parts_by_size = nvec / kResidualThreads > 0 ? nvec / kResidualThreads : 1;
+    if (parts > max_parts_by_size) parts = max_parts_by_size;
+    if (parts > kMaxResidualCtas) parts = kMaxResidualCtas;
+    if (parts < 1) parts = 1;
+    G.residual_ctas = parts;
+    *out = G;
+    return true;
+}
+
+struct WorkspaceLayout {
+    size_t partials, tasks, candidates, total;
+};
+static size_t round256(size_t n) { return (n + 255) & ~static_cast<size_t>(255); }
+static WorkspaceLayout layout_of(const Geometry& G) {
+    WorkspaceLayout L;
+    L.partials = 0;
+    L.tasks = round256(static_cast<size_t>(G.num_units) * G.max_slots * kConsumerWarps * sizeof(Partial));
+    L.candidates = L.tasks + round256(static_cast<size_t>(G.B) * sizeof(ResidualTask));
+    L.total = L.candidates + round256(static_cast<size_t>(G.B) * kMaxResidualCtas * 2 * sizeof(Candidate));
+    return L;
+}
+
+template <typename Kernel>
+static cudaError_t allow_large_smem(Kernel k, int dev, int which, size_t bytes) {
+    if (g_attr_done[dev][which]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e == cudaSuccess) g_attr_done[dev][which] = true;
+    return e;
+}
+
+template <int DT, bool GREEDY>
+static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream) {
+    const Geometry& G = P.geo;
+    const size_t smem = static_cast<size_t>(kStages) * kTileBytes + 2 * kStages * sizeof(uint64_t) + 16;
+    if (G.num_tiles > 0) {
+        cudaError_t e = allow_large_smem(stream_kernel<DT, GREEDY>, dev, DT * 2 + (GREEDY ? 1 : 0), smem);
+        if (e != cudaSuccess) return e;
+        stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, smem, stream>>>(P);
+    }
+    scan_kernel<DT, GREEDY><<<G.B, kScanWarps * 32, 0, stream>>>(P);
+    if (!GREEDY) residual_kernel<DT><<<dim3(G.residual_ctas, G.B), kResidualThreads, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+}  // namespace fef
+
+extern "C" {
+
+const char* fef_status_string(fef_status s) {
+    switch (s) {
+        case FEF_OK: return "ok";
+        case FEF_ERR_INVALID_ARG: return "invalid argument";
+        case FEF_ERR_DTYPE: return "unsupported dtype";
+        case FEF_ERR_ALIGNMENT: return "logit pointer or row pitch not a multiple of 16 bytes";
+        case FEF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case FEF_ERR_CUDA: return "CUDA error or no CUDA device";
+        case FEF_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case FEF_ERR_NONFINITE: return "NaN or +inf logit, or a row of -inf only";
+        case FEF_ERR_TOKEN_RANGE: return "draft token outside [0, V)";
+    }
+    return "unknown status";
+}
+
+size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
+    const int sms = fef::sm_count_of_current_device(nullptr);
+    fef::Geometry sampling, greedy;
+    if (!fef::make_geometry(B, K, V, V, dt, false, sms, &sampling)) return 0;
+    if (!fef::make_geometry(B, K, V, V, dt, true, sms, &greedy)) return 0;
+    const size_t a = fef::layout_of(sampling).total, b = fef::layout_of(greedy).total;
+    return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
+}
+
+fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* cuda_stream) {
+    using namespace fef;
+    if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
+    if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
+        return FEF_ERR_INVALID_ARG;
+    if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V) return FEF_ERR_INVALID_ARG;
+    if (!(temperature >= 0.0f) || isinf(temperature)) return FEF_ERR_INVALID_ARG;
+    const int esize = dt == FEF_F32 ? 4 : 2;
+    if (static_cast<int64_t>(V) * esize > (1ll << 30)) return FEF_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(draft_logits) & 15) || (reinterpret_cast<uintptr_t>(target_logits) & 15) ||
+        ((ld * esize) & 15))
+        return FEF_ERR_ALIGNMENT;
+
+    int dev = 0;
+    const int sms = sm_count_of_current_device(&dev);
+    if (sms < 1) return FEF_ERR_CUDA;
+    const bool greedy = (temperature == 0.0f);
+
+    VerifyParams P;
+    if (!make_geometry(B, K, V, ld, dt, greedy, sms, &P.geo)) return FEF_ERR_INVALID_ARG;
+    const WorkspaceLayout L = layout_of(P.geo);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
+        return FEF_ERR_WORKSPACE;
+
+    // c = log2(e) / T as c_hi + c_lo with c_lo > 0 (greedy mode reports T = 1 confidences)
+    const double c = 1.4426950408889634074 / (greedy ? 1.0 : static_cast<double>(temperature));
+    float c_hi = static_cast<float>(c);
+    if (static_cast<double>(c_hi) >= c) c_hi = nextafterf(c_hi, 0.0f);
+    P.c_hi = c_hi;
+    P.c_lo = static_cast<float>(c - static_cast<double>(c_hi));
+    if (!(P.c_hi > 0.f) || !(P.c_lo > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
+
+    P.target = static_cast<const char*>(target_logits);
+    P.draft = static_cast<const char*>(draft_logits);
+    P.draft_tokens = draft_tokens;
+    P.row_len = row_len;
+    P.seed = seed;
+    P.step = step;
+    P.accept_len = accept_len;
+    P.tokens = tokens;
+    P.conf = conf;
+    char* ws = static_cast<char*>(workspace);
+    P.partials = reinterpret_cast<Partial*>(ws + L.partials);
+    P.tasks = reinterpret_cast<ResidualTask*>(ws + L.tasks);
+    P.candidates = reinterpret_cast<Candidate*>(ws + L.candidates);
+    P.status = device_status;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (device_status && cudaMemsetAsync(device_status, 0, sizeof(int32_t), stream) != cudaSuccess)
+        return FEF_ERR_CUDA;
+    cudaError_t e;
+    if (dt == FEF_F32)
+        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream) : launch_all<FEF_F32, false>(P, dev, stream);
+    else
+        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream) : launch_all<FEF_BF16, false>(P, dev, stream);
+    return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,82 @@
+"""Host-side driver of the paper's full-sequence decoding loop (Algorithm 2) around
+the two library calls, for tests and benchmarks.
+
+The models are replaced by a caller-supplied ``logits_fn`` that returns the draft
+and target logits of the current speculative windows; everything the paper's loop
+does besides the two library calls is bookkeeping on small integer arrays, kept
+on the host here:
+
+  for s = 0 .. n_steps-1:                       (denoising steps)
+      C <- {}                                   (positions committed during this step)
+      while some position is unresolved:        (speculative rounds)
+          window = first min(K, #unresolved) unresolved positions of each batch row
+          verify(window)  -> commit accepted drafts and the corrected token, record c_j
+      if s < n_steps-1: R = LowConf_k(C); re-mask the positions in R
+
+Re-corruption uses the absorbing-state forward kernel: a selected position goes
+back to [MASK] (stored as -1).  ``verify_fn`` and ``select_fn`` are injected so the
+same driver can run any implementation.
+"""
+from __future__ import annotations
+
+from typing import Callable, Optional
+
+import numpy as np
+import torch
+
+MASK = -1
+
+
+def run_decode_loop(B: int, L: int, K: int, n_steps: int, remask_k: int,
+                    logits_fn: Callable, draft_fn: Callable, verify_fn: Callable, select_fn: Callable,
+                    on_round: Optional[Callable] = None, device="cuda", first_round: int = 0):
+    """Run Algorithm 2 on ``B`` sequences of ``L`` positions that all start masked.
+
+    logits_fn(round, window_pos [B,K] int64 (-1 = unused), row_len [B]) -> (draft_logits, target_logits)  [B,K,V]
+    draft_fn(draft_logits, round) -> draft_tokens [B,K] int32
+    verify_fn(draft_logits, target_logits, draft_tokens, row_len int32 [B] tensor, round)
+        -> (accept_len [B], tokens [B,K], conf [B,K]) as host numpy arrays
+    select_fn(conf [B,L] float32 tensor, mask [B,L] uint8 tensor, k) -> (positions [B,k], count [B]) numpy
+    on_round(round, inputs, outputs): optional hook (parity checks)
+
+    Returns dict(tokens [B,L], conf [B,L], rounds, committed_per_round list).
+    """
+    tokens = np.full((B, L), MASK, dtype=np.int64)
+    conf = np.full((B, L), -1.0, dtype=np.float32)
+    rnd = first_round
+    committed_hist = []
+    for s in range(n_steps):
+        in_C = np.zeros((B, L), dtype=np.uint8)
+        while (tokens == MASK).any():
+            window = np.full((B, K), -1, dtype=np.int64)
+            row_len = np.zeros(B, dtype=np.int32)
+            for b in range(B):
+                unresolved = np.nonzero(tokens[b] == MASK)[0][:K]
+                row_len[b] = len(unresolved)
+                window[b, :len(unresolved)] = unresolved
+            q, p = logits_fn(rnd, window, row_len)
+            draft = draft_fn(q, rnd)
+            rl = torch.as_tensor(row_len, device=device)
+            accept_len, out_tok, out_conf = verify_fn(q, p, draft, rl, rnd)
+            if on_round is not None:
+                on_round(rnd, (q, p, draft, rl), (accept_len, out_tok, out_conf))
+            n_committed = 0
+            for b in range(B):
+                if accept_len[b] < 0:
+                    raise RuntimeError("verification reported a data error in window %d" % b)
+                m = min(int(accept_len[b]) + 1, int(row_len[b]))
+                pos = window[b, :m]
+                tokens[b, pos] = out_tok[b, :m]
+                conf[b, pos] = out_conf[b, :m]
+                in_C[b, pos] = 1
+                n_committed += m
+            committed_hist.append(n_committed)
+            rnd += 1
+        if s < n_steps - 1 and remask_k > 0:
+            positions, count = select_fn(torch.as_tensor(conf, device=device), torch.as_tensor(in_C, device=device),
+                                         remask_k)
+            for b in range(B):
+                sel = positions[b, :count[b]]
+                tokens[b, sel] = MASK
+                conf[b, sel] = -1.0
+    return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist)

@@ -1,0 +1,299 @@
+"""CUDA library against the CPU oracle, element by element, through the C ABI (needs a B200)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle.compare import ParityReport, compare_verify
+from paper_2605_14305_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fef():
+    import paper_2605_14305_b200 as lib
+
+    lib.load(build_if_missing=True)
+    return lib
+
+
+def _gpu_verify(fef, q, p, tok, T, seed, step, row_len=None, V=None):
+    r = fef.fef_spec_verify(q, p, tok, T, seed, step, row_len=row_len, V=V)
+    torch.cuda.synchronize()
+    return (r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy(), int(r.device_status.item()))
+
+
+def _check(fef, q, p, tok, T, seed, step, row_len=None, V=None, expect_status=0) -> ParityReport:
+    """q, p, tok: CUDA tensors.  Runs both sides on the same bytes and compares."""
+    ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, T, seed, step, row_len, V)
+    ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), T, seed, step,
+                             row_len=None if row_len is None else row_len.cpu(), V=V)
+    assert ref["status"] == expect_status
+    assert gs == expect_status
+    rep = compare_verify(ga, gt, gc, ref)
+    assert rep.ok, rep.mismatches[:5]
+    return rep
+
+
+def _random_case(B, K, V, dtype, noise, seed, ld=None, scale=2.0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    ld = V if ld is None else ld
+    q = torch.randn((B, K, ld), generator=g, device="cuda") * scale
+    p = q + torch.randn((B, K, ld), generator=g, device="cuda") * noise
+    q, p = q.to(dtype), p.to(dtype)
+    if ld > V:  # padding must never be read
+        q[:, :, V:] = float("nan")
+        p[:, :, V:] = float("inf")
+    tok = synth.sample_draft_tokens(q[:, :, :V].contiguous(), 1.0, seed + 1)
+    return q, p, tok
+
+
+SMALL_SHAPES = [
+    # B, K, V, ld
+    (1, 1, 1, 4), (2, 3, 3, 4), (3, 2, 4, 4), (2, 4, 7, 8), (5, 4, 8, 8), (2, 5, 9, 12), (3, 7, 33, 36),
+    (4, 4, 1000, 1000), (1, 4, 1024, 1024), (2, 3, 4097, 4104), (7, 32, 260, 264), (2, 64, 520, 520),
+    (300, 2, 64, 64), (2, 2, 40000, 40000), (1, 3, 70001, 70008),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T", [1.0, 0.7, 0.0])
+def test_small_shapes_match_oracle(fef, dtype, T):
+    total = ParityReport()
+    for n, (B, K, V, ld) in enumerate(SMALL_SHAPES):
+        if dtype == torch.bfloat16:
+            ld = (ld + 7) // 8 * 8
+        q, p, tok = _random_case(B, K, V, dtype, 0.8, 100 + n, ld=ld)
+        if T == 0.0:  # make most drafts the arg-max so windows get past position 0
+            top = p[:, :, :V].float().argmax(-1).to(torch.int32)
+            keep = torch.rand(tok.shape, device="cuda") < 0.3
+            tok = torch.where(keep, tok, top)
+        total.merge(_check(fef, q, p, tok, T, seed=7 + n, step=n, V=V))
+    print(total.summary())
+    assert total.excused <= 1
+
+
+def test_tiny_config_decode_loop_100_steps(fef):
+    """Config 0: B=1, K=4, V=1024, fp32, T=1, re-mask k=2; every call checked against the oracle."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop
+
+    w = synth.TINY
+    total = ParityReport()
+
+    def logits_fn(rnd, window, row_len):
+        return synth.make_logits(w, seed=1000 + rnd, device="cuda")
+
+    def draft_fn(q, rnd):
+        return synth.sample_draft_tokens(q, w.temperature, 5000 + rnd)
+
+    def verify_fn(q, p, tok, rl, rnd):
+        ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, w.temperature, 0, rnd, row_len=rl)
+        assert gs == 0
+        ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), w.temperature, 0, rnd, row_len=rl.cpu())
+        rep = compare_verify(ga, gt, gc, ref)
+        assert rep.ok, rep.mismatches
+        total.merge(rep)
+        return ga, gt, gc
+
+    def select_fn(conf, mask, k):
+        pos, cnt = fef.fef_remask_select(conf, mask, k)
+        opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
+        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
+        return opos, ocnt
+
+    out = run_decode_loop(w.B, w.gen_len, w.K, 100, w.remask_k, logits_fn, draft_fn, verify_fn, select_fn)
+    assert (out["tokens"] >= 0).all()
+    assert out["rounds"] >= 100
+    print(total.summary(), "rounds", out["rounds"])
+
+
+def test_llada_single_stream_block(fef):
+    """Config 1 (B=1, K=32, V=126464, bf16, peaked logits): one block, three denoising steps,
+    every call checked; the row is split over many CTAs here."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop
+
+    w = synth.LLADA_SINGLE
+    total = ParityReport()
+
+    def logits_fn(rnd, window, row_len):
+        return synth.make_logits(w, seed=2000 + rnd, device="cuda")
+
+    def draft_fn(q, rnd):
+        return synth.sample_draft_tokens(q, w.temperature, 6000 + rnd)
+
+    def verify_fn(q, p, tok, rl, rnd):
+        ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, w.temperature, 11, rnd, row_len=rl)
+        assert gs == 0
+        ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), w.temperature, 11, rnd, row_len=rl.cpu())
+        rep = compare_verify(ga, gt, gc, ref)
+        assert rep.ok, rep.mismatches
+        total.merge(rep)
+        return ga, gt, gc
+
+    def select_fn(conf, mask, k):
+        pos, cnt = fef.fef_remask_select(conf, mask, k)
+        opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
+        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
+        return opos, ocnt
+
+    out = run_decode_loop(w.B, w.K, w.K, 3, w.remask_k, logits_fn, draft_fn, verify_fn, select_fn)
+    assert (out["tokens"] >= 0).all()
+    print(total.summary(), "rounds", out["rounds"])
+
+
+@pytest.mark.parametrize("sigma", [0.2, 0.7, 1.5])
+def test_llada_batched_sigma_sweep(fef, sigma):
+    """Config 2: B=16, K=32, V=126464, bf16, T=0.7; the noise level moves the acceptance rate."""
+    w = synth.LLADA_BATCHED
+    q, p, tok = synth.make_call(w, seed=int(sigma * 100), device="cuda", noise_std=sigma)
+    rep = _check(fef, q, p, tok, w.temperature, seed=3, step=int(sigma * 10))
+    ga, _, gc, _ = _gpu_verify(fef, q, p, tok, w.temperature, 3, int(sigma * 10))
+    print("sigma", sigma, rep.summary(), "mean accept_len", ga.mean())
+    # the re-mask selection of this configuration (k = 8) on the confidences just produced
+    mask = torch.as_tensor(gc >= 0).to(torch.uint8).cuda()
+    pos, cnt = fef.fef_remask_select(torch.as_tensor(gc).cuda(), mask, w.remask_k)
+    opos, ocnt = oracle.remask_select(gc, mask.cpu(), w.remask_k)
+    assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
+
+
+@pytest.mark.parametrize("T", [1.0, 0.0])
+def test_dream_large_batch_sampled_windows(fef, T):
+    """Config 3 at full size (B=64, K=32, V=152064, bf16, Zipf-biased logits) in the launch
+    configuration the benchmark uses; the oracle re-computes a sample of whole windows."""
+    w = synth.DREAM_LARGE.with_(temperature=T)
+    q, p, tok = synth.make_call(w, seed=33, device="cuda")
+    if T == 0.0:
+        top = p.float().argmax(-1).to(torch.int32)
+        tok = torch.where(torch.rand(tok.shape, device="cuda") < 0.15, tok, top)
+    ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, T, 17, 4)
+    assert gs == 0
+    total = ParityReport()
+    for b in (0, 1, 13, 31, 62, 63):
+        ref = oracle.spec_verify(q[b:b + 1].cpu(), p[b:b + 1].cpu(), tok[b:b + 1].cpu(), T, 17, 4, batch_offset=b)
+        rep = compare_verify(ga[b:b + 1], gt[b:b + 1], gc[b:b + 1], ref, batch_offset=b)
+        assert rep.ok, rep.mismatches
+        total.merge(rep)
+    # properties that hold for every window at any size
+    K = w.K
+    assert ((ga >= 0) & (ga <= K)).all()
+    idx = np.arange(K)[None, :]
+    committed = idx < np.minimum(ga + 1, K)[:, None]
+    assert ((gt >= 0) == committed).all() and ((gc >= 0) == committed).all()
+    accepted = idx < ga[:, None]
+    assert (gt[accepted] == tok.cpu().numpy()[accepted]).all()
+    assert (gc[committed] <= 1.0 + 1e-6).all()
+    print(total.summary(), "mean accept_len", ga.mean())
+
+
+def test_headline_shape_sampled_windows(fef):
+    """The benchmark's workload (B=64, K=32, V=126464, bf16, T=1) with sampled windows checked."""
+    w = synth.HEADLINE
+    q, p, tok = synth.make_call(w, seed=5, device="cuda")
+    ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, w.temperature, 99, 1)
+    assert gs == 0
+    total = ParityReport()
+    for b in (0, 7, 40, 63):
+        ref = oracle.spec_verify(q[b:b + 1].cpu(), p[b:b + 1].cpu(), tok[b:b + 1].cpu(), w.temperature, 99, 1,
+                                 batch_offset=b)
+        rep = compare_verify(ga[b:b + 1], gt[b:b + 1], gc[b:b + 1], ref, batch_offset=b)
+        assert rep.ok, rep.mismatches
+        total.merge(rep)
+    print(total.summary(), "mean accept_len", ga.mean())
+
+
+def test_results_are_bit_identical_across_runs(fef):
+    q, p, tok = _random_case(8, 16, 30000, torch.bfloat16, 0.9, 77)
+    a = _gpu_verify(fef, q, p, tok, 0.9, 5, 6)
+    for _ in range(3):
+        b = _gpu_verify(fef, q, p, tok, 0.9, 5, 6)
+        assert (a[0] == b[0]).all() and (a[1] == b[1]).all() and (a[2] == b[2]).all()
+
+
+def test_identical_laws_accept_everything(fef):
+    q, _, tok = _random_case(6, 32, 5000, torch.bfloat16, 0.5, 5)
+    rep = _check(fef, q, q.clone(), tok, 0.8, 1, 1)
+    ga, gt, _, _ = _gpu_verify(fef, q, q.clone(), tok, 0.8, 1, 1)
+    assert (ga == 32).all() and (gt == tok.cpu().numpy()).all()
+
+
+def test_row_len_and_empty_windows(fef):
+    q, p, tok = _random_case(9, 8, 3000, torch.float32, 0.3, 9)
+    row_len = torch.tensor([0, 1, 8, 3, 0, 8, 7, 2, 5], dtype=torch.int32, device="cuda")
+    # garbage beyond row_len must not matter
+    tok2 = tok.clone()
+    for b in range(9):
+        tok2[b, int(row_len[b]):] = -12345
+        p[b, int(row_len[b]):] = float("nan")
+    _check(fef, q, p, tok2, 1.0, 4, 4, row_len=row_len)
+
+
+def test_minus_inf_and_zero_probability_conventions(fef):
+    B, K, V = 4, 2, 64
+    q, p, tok = _random_case(B, K, V, torch.float32, 0.5, 21)
+    q[0, 0, 5] = -math.inf; tok[0, 0] = 5                         # rho(x)=0 < pi(x): accept
+    q[1, 0, 6] = -math.inf; p[1, 0, 6] = -math.inf; tok[1, 0] = 6   # pi=rho=0: reject, residual draw
+    p[2, 1, 10:40] = -math.inf                                     # masked vocabulary range
+    q[3, 0] = p[3, 0]; p[3, 0, 9] = -math.inf; q[3, 0, 9] = -math.inf; tok[3, 0] = 9  # reject with zero residual
+    rep = _check(fef, q, p, tok, 1.0, 8, 8)
+    ga, gt, _, _ = _gpu_verify(fef, q, p, tok, 1.0, 8, 8)
+    assert ga[0] >= 1 and ga[1] == 0 and ga[3] == 0
+    assert gt[3, 0] == int(p[3, 0].argmax())
+
+
+def test_data_errors_set_status_and_poison_only_their_window(fef):
+    q, p, tok = _random_case(5, 4, 2000, torch.bfloat16, 0.5, 31)
+    bad = p.clone(); bad[1, 2, 1234] = float("nan")
+    _check(fef, q, bad, tok, 1.0, 1, 1, expect_status=7)
+    bad = q.clone(); bad[2, 0, 0] = float("inf")
+    _check(fef, bad, p, tok, 1.0, 1, 1, expect_status=7)
+    bad = p.clone(); bad[4, 3, :] = -math.inf
+    _check(fef, q, bad, tok, 1.0, 1, 1, expect_status=7)
+    t2 = tok.clone(); t2[0, 1] = 2000
+    _check(fef, q, p, t2, 1.0, 1, 1, expect_status=8)
+    t2 = tok.clone(); t2[3, 0] = -1
+    _check(fef, q, p, t2, 0.0, 1, 1, expect_status=8)
+    # a later clean call resets the status word
+    _check(fef, q, p, tok, 1.0, 1, 1, expect_status=0)
+
+
+def test_far_apart_laws_reject_at_once_and_wide_dynamic_range(fef):
+    g = torch.Generator(device="cuda").manual_seed(3)
+    B, K, V = 3, 4, 9000
+    q = torch.randn((B, K, V), generator=g, device="cuda") * 30.0      # logits spanning +-100
+    p = torch.randn((B, K, V), generator=g, device="cuda") * 30.0
+    tok = synth.sample_draft_tokens(q, 1.0, 4)
+    _check(fef, q, p, tok, 1.0, 2, 2)
+    _check(fef, q + 500.0, p - 500.0, tok, 1.0, 2, 3)                  # large common offsets
+    # increasing ramp: the running reference has to move many times
+    ramp = torch.linspace(-200, 200, V, device="cuda").expand(B, K, V).contiguous()
+    _check(fef, ramp, (ramp * 0.98).contiguous(), tok, 1.0, 2, 4)
+
+
+@pytest.mark.parametrize("B,L,k", [(1, 1, 1), (3, 17, 5), (8, 256, 8), (2, 1024, 2), (4, 33, 40), (2, 9, 0),
+                                   (2, 8192, 8), (64, 1024, 8), (1, 5000, 5000)])
+def test_remask_select_matches_oracle(fef, B, L, k):
+    g = torch.Generator(device="cuda").manual_seed(B * 1000 + L)
+    conf = torch.rand((B, L), generator=g, device="cuda")
+    conf[torch.rand((B, L), generator=g, device="cuda") < 0.3] = 0.25     # many exact ties
+    conf[torch.rand((B, L), generator=g, device="cuda") < 0.05] = -1.0    # sentinels
+    conf[torch.rand((B, L), generator=g, device="cuda") < 0.02] = 0.0
+    conf[torch.rand((B, L), generator=g, device="cuda") < 0.02] = -0.0
+    mask = (torch.rand((B, L), generator=g, device="cuda") < 0.6).to(torch.uint8)
+    if B > 1:
+        mask[1] = 0
+    pos, cnt = fef.fef_remask_select(conf, mask, k)
+    torch.cuda.synchronize()
+    opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
+    assert (cnt.cpu().numpy() == ocnt).all()
+    assert (pos.cpu().numpy() == opos).all()
+
+
+def test_remask_select_nan_sorts_last(fef):
+    conf = torch.tensor([[0.5, float("nan"), 0.1, float("inf"), float("nan"), -1.0]], device="cuda")
+    mask = torch.ones_like(conf, dtype=torch.uint8)
+    pos, cnt = fef.fef_remask_select(conf, mask, 6)
+    opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), 6)
+    assert pos.cpu().numpy().tolist() == opos.tolist() == [[5, 2, 0, 3, 1, 4]]

@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-verification hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input:
+``fef_spec_verify`` (streaming softmax statistics, acceptance scan, residual
+draw, confidences) followed by ``fef_remask_select`` (LowConf_k).  The workload
+is the headline configuration: B = 64 windows of K = 32 draft positions,
+V = 126464 (LLaDA-8B vocabulary), bf16 logits, temperature 1, peaked synthetic
+logits with target = draft + N(0, 0.7^2); the re-mask selection runs on a
+[64, 1024] confidence state with k = 8.
+
+Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on the
+host cores instead (a deliberately slow program; context, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_14305_b200 import synth  # noqa: E402
+
+METRIC = "verified draft positions/sec"
+UNIT = "positions/s"
+REMASK_L = 1024
+FALLBACK_HBM_GBS = 6650.0
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "stream_kernel_headline_bf16.txt")
+
+
+# ------------------------------------------------------------------ helpers ----
+def _workload(args) -> synth.Workload:
+    w = synth.CONFIGS[args.workload]
+    over = {}
+    for name in ("B", "K", "V"):
+        if getattr(args, name) is not None:
+            over[name] = getattr(args, name)
+    if args.dtype is not None:
+        over["dtype"] = torch.float32 if args.dtype == "f32" else torch.bfloat16
+    if args.temperature is not None:
+        over["temperature"] = args.temperature
+    if args.noise is not None:
+        over["noise_std"] = args.noise
+    return w.with_(**over) if over else w
+
+
+def _config_dict(w: synth.Workload, extra=None):
+    cfg = {
+        "workload": "%s: B=%d windows x K=%d draft positions, V=%d, %s logits, T=%g, %s draft logits, "
+                    "target = draft + N(0, %g^2); re-mask select on [%d, %d] confidences, k=%d"
+                    % (w.name, w.B, w.K, w.V, "bf16" if w.dtype == torch.bfloat16 else "fp32", w.temperature,
+                       w.family, w.noise_std, w.B, REMASK_L, w.remask_k),
+        "B": w.B, "K": w.K, "V": w.V, "temperature": w.temperature, "remask_k": w.remask_k,
+        "l2": "inputs of one step (%s) exceed the 126 MB L2 and two input sets alternate"
+              % synth.human_bytes(synth.algorithmic_bytes(w)),
+    }
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def _measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def _ncu_traffic():
+    """DRAM bytes per launch of the streaming kernel from the committed ncu summary, or None."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                if line.startswith("traffic_bytes_per_launch:"):
+                    return float(line.split(":", 1)[1].split()[0])
+    except Exception:
+        pass
+    return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            handle = None
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.handle = handle
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def sample(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+            try:
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+            except Exception:
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+            for bit, name in self.REASONS.items():
+                if bits & bit:
+                    self.reasons.add(name)
+            self.power.append(nv.nvmlDeviceGetPowerUsage(self.handle) / 1000.0)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._halt.is_set():
+            self.sample()
+            self._halt.wait(self.period)
+
+    def stop(self):
+        self.sample()
+        self._halt.set()
+
+    def result(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None}
+
+
+# ------------------------------------------------------------- native arm ----
+def run_native(args):
+    import torch.distributed as dist
+
+    import paper_2605_14305_b200 as fef
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the native arm has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    fef.load(build_if_missing=True)
+
+    w = _workload(args)
+    steps, warmup = args.steps, max(args.warmup, 3)
+    nbuf = 2
+    sets = [synth.make_call(w, seed=1000 * (rank + 1) + i, device=dev) for i in range(nbuf)]
+    g = torch.Generator(device=dev).manual_seed(77 + rank)
+    conf_state = torch.rand((w.B, REMASK_L), generator=g, device=dev)
+    mask_state = (torch.rand((w.B, REMASK_L), generator=g, device=dev) < 0.5).to(torch.uint8)
+    out = fef.VerifyResult(torch.empty(w.B, dtype=torch.int32, device=dev),
+                           torch.empty((w.B, w.K), dtype=torch.int32, device=dev),
+                           torch.empty((w.B, w.K), dtype=torch.float32, device=dev),
+                           torch.zeros(1, dtype=torch.int32, device=dev))
+    ws = torch.empty(max(fef.fef_spec_verify_workspace_bytes(w.B, w.K, w.V, w.dtype), 256), dtype=torch.uint8,
+                     device=dev)
+    positions = torch.empty((w.B, w.remask_k), dtype=torch.int32, device=dev)
+    count = torch.empty(w.B, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    for evs in stage_ev:
+        for e in evs:
+            e.record(stream)  # creates the underlying CUDA event
+
+    def step(i, events=None):
+        q, p, tok = sets[i % nbuf]
+        fef.fef_spec_verify(q, p, tok, w.temperature, args.seed, i, out=out, workspace=ws, stage_events=events)
+        fef.fef_remask_select(conf_state, mask_state, w.remask_k, positions=positions, count=count)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        step(warmup + i, stage_ev[i] if not args.no_stage_events else None)
+    t1.record(stream)
+    barrier()
+    sampler.stop()
+    elapsed_ms = t0.elapsed_time(t1)
+    status = int(out.device_status.item())
+    accept_mean = float(out.accept_len.float().mean().item())
+    rejected = int((out.accept_len < w.K).sum().item())
+
+    stage_ms = [0.0, 0.0, 0.0]
+    if not args.no_stage_events:
+        for evs in stage_ev:
+            for j in range(3):
+                stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
+        stage_ms = [x / steps for x in stage_ms]
+
+    # ---- end to end through the host-buffer entry points (copies inside the timed region)
+    e2e_steps = max(1, min(steps, args.e2e_steps))
+    hq, hp, htok = (t.cpu().pin_memory() for t in sets[0])
+    hconf, hmask = conf_state.cpu().pin_memory(), mask_state.cpu().pin_memory()
+    arena = torch.empty(fef.fef_spec_verify_host_arena_bytes(w.B, w.K, w.V, w.V, w.dtype), dtype=torch.uint8, device=dev)
+    arena2 = torch.empty(fef.fef_remask_select_host_arena_bytes(w.B, REMASK_L, w.remask_k), dtype=torch.uint8, device=dev)
+    hout = fef.HostVerifyResult(torch.empty(w.B, dtype=torch.int32).pin_memory(),
+                                torch.empty((w.B, w.K), dtype=torch.int32).pin_memory(),
+                                torch.empty((w.B, w.K), dtype=torch.float32).pin_memory(), 0)
+    hpos = torch.empty((w.B, w.remask_k), dtype=torch.int32).pin_memory()
+    hcnt = torch.empty(w.B, dtype=torch.int32).pin_memory()
+
+    def host_step(i):
+        fef.fef_spec_verify_host(hq, hp, htok, w.temperature, args.seed, i, arena, out=hout)
+        fef.fef_remask_select_host(hconf, hmask, w.remask_k, arena2, positions=hpos, count=hcnt)
+
+    host_step(0)
+    barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record(stream)
+    for i in range(e2e_steps):
+        host_step(1 + i)
+    h1.record(stream)
+    barrier()
+    e2e_ms = h0.elapsed_time(h1)
+
+    if world > 1:
+        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+
+    logits_bytes = hq.numel() * hq.element_size() * (2 if w.temperature > 0 else 1)
+    h2d = logits_bytes + htok.numel() * 4 + hconf.numel() * 4 + hmask.numel()
+    d2h = w.B * 4 + w.B * w.K * 8 + 4 + w.B * w.remask_k * 4 + w.B * 4
+
+    # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only
+    cpu_baseline, parity = None, None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        from oracle.compare import compare_verify
+
+        nwin = min(w.B, args.cpu_windows)
+        q, p, tok = (t[:nwin].cpu() for t in sets[0])
+        reps, t_cpu, ref = 0, 0.0, None
+        while t_cpu < args.cpu_seconds and reps < 8:
+            c0 = time.perf_counter()
+            ref = oracle.spec_verify(q, p, tok, w.temperature, args.seed, 424242)
+            t_cpu += time.perf_counter() - c0
+            reps += 1
+        cpu_baseline = {"value": reps * nwin * w.K / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "host_cores": os.cpu_count(),
+                        "sample": "%d call(s) over the first %d of %d windows of the same batch (%d positions each), "
+                                  "%.1f s of single-thread CPU time" % (reps, nwin, w.B, nwin * w.K, t_cpu)}
+        got = fef.fef_spec_verify(sets[0][0], sets[0][1], sets[0][2], w.temperature, args.seed, 424242)
+        torch.cuda.synchronize()
+        rep = compare_verify(got.accept_len[:nwin].cpu().numpy(), got.tokens[:nwin].cpu().numpy(),
+                             got.conf[:nwin].cpu().numpy(), ref)
+        parity = {"windows": rep.windows, "draws": rep.draws, "near_margin": rep.near_margin,
+                  "excused": rep.excused, "mismatches": len(rep.mismatches),
+                  "max_conf_rel_err": rep.max_conf_rel_err}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    positions_per_step = w.B * w.K * world
+    value = positions_per_step * steps / (elapsed_ms * 1e-3)
+    peak, peak_src = _measured_peak()
+    row_bytes = (2 if w.temperature > 0 else 1) * w.V * w.logit_bytes
+    stream_bytes = w.B * w.K * row_bytes
+    roof = {"bound": "hbm", "kernel": "stream_kernel", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
+            "traffic": _ncu_traffic(), "algorithmic_bytes_per_launch": stream_bytes}
+    if not args.no_stage_events and stage_ms[0] > 0:
+        roof["achieved"] = stream_bytes / (stage_ms[0] * 1e-3) / 1e9
+        roof["frac"] = roof["achieved"] / peak
+        roof["ms_per_launch"] = stage_ms[0]
+        roof["stage_ms"] = {"stream": stage_ms[0], "scan": stage_ms[1], "residual": stage_ms[2]}
+    else:
+        roof["achieved"], roof["frac"] = None, None
+    call_bytes = synth.algorithmic_bytes(w, rejected_rows=rejected)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": _config_dict(w, {"parallelism": "replicas x%d (windows are independent; no collective)" % world}),
+        "impl": "native",
+        "hbm_gbs_whole_step": call_bytes / (elapsed_ms / steps * 1e-3) / 1e9,
+        "frac_of_8TBs_whole_step": call_bytes / (elapsed_ms / steps * 1e-3) / 8e12,
+        "roofline": roof,
+        "e2e": {"value": positions_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "ms_per_step": e2e_ms / e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "api": "fef_spec_verify_host + fef_remask_select_host (pinned host buffers)"},
+        "gpu_launches": steps * 4,
+        "clocks": sampler.result(),
+        "cpu_baseline": cpu_baseline,
+        "parity_vs_oracle": parity,
+        "device_status": status, "mean_accept_len": accept_mean,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------- reference arm ----
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: each step verifies a bounded sample
+    (the first n windows) of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+
+    w = _workload(args)
+    steps, warmup = args.steps, args.warmup
+    # about 0.07 s of CPU time per headline-shaped window; keep the whole run near two minutes
+    per_window_s = 0.07 * (w.V / 126464.0) * (w.K / 32.0)
+    nwin = int(max(1, min(w.B, math.floor(120.0 / ((steps + warmup) * per_window_s)))))
+    q, p, tok = synth.make_call(w.with_(B=nwin), seed=1000, device="cpu")
+    for i in range(warmup):
+        oracle.spec_verify(q, p, tok, w.temperature, args.seed, i)
+    c0 = time.perf_counter()
+    for i in range(steps):
+        ref = oracle.spec_verify(q, p, tok, w.temperature, args.seed, warmup + i)
+        conf = ref["conf"].astype("float32")
+        oracle.remask_select(conf, (conf >= 0).astype("uint8"), w.remask_k)
+    elapsed = time.perf_counter() - c0
+    value = nwin * w.K * steps / elapsed
+    sample = "each step: the first %d of %d windows (%d positions) of the workload" % (nwin, w.B, nwin * w.K)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": elapsed / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config_dict(w, {"parallelism": "one host thread"}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["native", "reference"], default="native")
+    ap.add_argument("--workload", default="headline", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--B", type=int)
+    ap.add_argument("--K", type=int)
+    ap.add_argument("--V", type=int)
+    ap.add_argument("--dtype", choices=["bf16", "f32"])
+    ap.add_argument("--temperature", type=float)
+    ap.add_argument("--noise", type=float)
+    ap.add_argument("--seed", type=int, default=20260514)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-windows", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stage-events", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -111,6 +111,44 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
                            int32_t* device_status, void* cuda_stream);
 
 /*
+ * fef_spec_verify with timing marks: the same operation (Algorithm 2's verification
+ * loop), and additionally records up to four caller-created CUDA events
+ * (cudaEvent_t passed as void*; NULL entries are skipped) on `cuda_stream`:
+ * [0] before the streaming pass, [1] after it, [2] after the acceptance scan,
+ * [3] after the residual pass.  `stage_events` may be NULL.  Used to time the
+ * stages separately; results are identical to fef_spec_verify.
+ */
+fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const int32_t* row_len,
+                                    int B, int K, int V, int64_t ld, fef_dtype dt,
+                                    float temperature, uint64_t seed, uint32_t step,
+                                    int32_t* accept_len, int32_t* tokens, float* conf,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* device_status, void* cuda_stream,
+                                    void* const* stage_events);
+
+/*
+ * Host-buffer form of fef_spec_verify (same operation, same citations): every
+ * array argument is HOST memory (pinned memory makes the copies asynchronous and
+ * fast).  The call copies the inputs into `device_arena`, runs the verification
+ * there, copies accept_len / tokens / conf and the device status word back, and
+ * returns after synchronising `cuda_stream`.  At temperature 0 the draft logits
+ * are not copied.
+ *   device_arena        device scratch, 256-byte aligned, at least
+ *                       fef_spec_verify_host_arena_bytes(B, K, V, ld, dt) bytes
+ *   status_out          host out, may be NULL: the device status word of the call
+ * The arena size is 0 for invalid sizes or when no CUDA device is available.
+ */
+size_t fef_spec_verify_host_arena_bytes(int B, int K, int V, int64_t ld, fef_dtype dt);
+fef_status fef_spec_verify_host(const void* draft_logits, const void* target_logits,
+                                const int32_t* draft_tokens, const int32_t* row_len,
+                                int B, int K, int V, int64_t ld, fef_dtype dt,
+                                float temperature, uint64_t seed, uint32_t step,
+                                int32_t* accept_len, int32_t* tokens, float* conf,
+                                int32_t* status_out,
+                                void* device_arena, size_t device_arena_bytes, void* cuda_stream);
+
+/*
  * LowConf_k of Algorithm 2 ("Select R = LowConf_{n_rm}(C)"): for every batch
  * row the k candidate positions of lowest confidence.
  *
@@ -124,6 +162,17 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
  */
 fef_status fef_remask_select(const float* conf, const uint8_t* mask, int B, int L, int k,
                              int32_t* positions, int32_t* count, void* cuda_stream);
+
+/*
+ * Host-buffer form of fef_remask_select (same operation): conf, mask, positions
+ * and count are HOST memory; the call stages them through `device_arena`
+ * (256-byte aligned, at least fef_remask_select_host_arena_bytes(B, L, k) bytes)
+ * and returns after synchronising `cuda_stream`.
+ */
+size_t fef_remask_select_host_arena_bytes(int B, int L, int k);
+fef_status fef_remask_select_host(const float* conf, const uint8_t* mask, int B, int L, int k,
+                                  int32_t* positions, int32_t* count,
+                                  void* device_arena, size_t device_arena_bytes, void* cuda_stream);
 
 #ifdef __cplusplus
 }

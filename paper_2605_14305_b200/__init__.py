@@ -21,7 +21,9 @@ FEF_ERR_CUDA, FEF_ERR_TIMEOUT, FEF_ERR_NONFINITE, FEF_ERR_TOKEN_RANGE = 5, 6, 7,
 FEF_F32, FEF_BF16 = 0, 1
 FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
 
-EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_remask_select")
+EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_spec_verify_profiled",
+           "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
+           "fef_remask_select_host_arena_bytes", "fef_remask_select_host")
 
 _lib = None
 
@@ -53,8 +55,18 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_workspace_bytes.restype = sz
     L.fef_spec_verify.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, sz, vp, vp]
     L.fef_spec_verify.restype = i32
+    L.fef_spec_verify_profiled.argtypes = L.fef_spec_verify.argtypes + [vp]
+    L.fef_spec_verify_profiled.restype = i32
+    L.fef_spec_verify_host_arena_bytes.argtypes = [i32, i32, i32, i64, i32]
+    L.fef_spec_verify_host_arena_bytes.restype = sz
+    L.fef_spec_verify_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp, sz, vp]
+    L.fef_spec_verify_host.restype = i32
     L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.fef_remask_select.restype = i32
+    L.fef_remask_select_host_arena_bytes.argtypes = [i32, i32, i32]
+    L.fef_remask_select_host_arena_bytes.restype = sz
+    L.fef_remask_select_host.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
+    L.fef_remask_select_host.restype = i32
     _lib = L
     return L
 
@@ -99,8 +111,12 @@ class VerifyResult(NamedTuple):
 def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, draft_tokens: torch.Tensor,
                     temperature: float, seed: int, step: int, row_len: Optional[torch.Tensor] = None,
                     V: Optional[int] = None, out: Optional[VerifyResult] = None,
-                    workspace: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+                    workspace: Optional[torch.Tensor] = None, stream=None, stage_events=None) -> VerifyResult:
     """Enqueue one verification call (see ``fef_spec_verify`` in include/fef.h).
+
+    With ``stage_events`` (four ``torch.cuda.Event(enable_timing=True)`` that have
+    been recorded once, or ``None`` entries) the call goes through
+    ``fef_spec_verify_profiled`` and the events mark the stage boundaries.
 
     ``draft_logits`` / ``target_logits``: ``[B, K, ld]`` CUDA tensors, float32 or
     bfloat16, contiguous; ``V`` (default ``ld``) entries of each row are used.
@@ -127,12 +143,16 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
         if workspace is None:
             workspace = torch.empty(max(fef_spec_verify_workspace_bytes(B, K, V, code), 256),
                                     dtype=torch.uint8, device=dev)
-        st = load().fef_spec_verify(
-            draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
-            None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
-            int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
-            out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
-            workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(), _stream_ptr(stream))
+        args = (draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
+                None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
+                int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
+                out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
+                workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(), _stream_ptr(stream))
+        if stage_events is None:
+            st = load().fef_spec_verify(*args)
+        else:
+            handles = (ctypes.c_void_p * 4)(*[None if e is None else e.cuda_event for e in stage_events])
+            st = load().fef_spec_verify_profiled(*args, handles)
     if st != FEF_OK:
         raise FefError(st, "fef_spec_verify")
     return out
@@ -167,5 +187,76 @@ def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions:
     return positions, count
 
 
-__all__ = ["load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
+def fef_spec_verify_host_arena_bytes(B: int, K: int, V: int, ld: int, dtype) -> int:
+    code = dtype if isinstance(dtype, int) else (FEF_F32 if dtype == torch.float32 else FEF_BF16)
+    return int(load().fef_spec_verify_host_arena_bytes(B, K, V, ld, code))
+
+
+class HostVerifyResult(NamedTuple):
+    accept_len: torch.Tensor  # host tensors
+    tokens: torch.Tensor
+    conf: torch.Tensor
+    status: int
+
+
+def fef_spec_verify_host(draft_logits: torch.Tensor, target_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                         temperature: float, seed: int, step: int, arena: torch.Tensor,
+                         row_len: Optional[torch.Tensor] = None, V: Optional[int] = None,
+                         out: Optional[HostVerifyResult] = None, stream=None) -> HostVerifyResult:
+    """Host-buffer form (see ``fef_spec_verify_host`` in include/fef.h): inputs and outputs are
+    CPU tensors (pin them for speed), ``arena`` is a CUDA uint8 tensor of at least
+    ``fef_spec_verify_host_arena_bytes`` bytes.  Returns after the results are on the host."""
+    _require_cuda(arena)
+    for t in (draft_logits, target_logits, draft_tokens, row_len):
+        if t is not None and (t.device.type != "cpu" or not t.is_contiguous()):
+            raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_host")
+    B, K, ld = draft_logits.shape
+    V = ld if V is None else int(V)
+    code = _dtype_code(draft_logits)
+    if out is None:
+        out = HostVerifyResult(torch.empty(B, dtype=torch.int32).pin_memory(),
+                               torch.empty((B, K), dtype=torch.int32).pin_memory(),
+                               torch.empty((B, K), dtype=torch.float32).pin_memory(), 0)
+    status = ctypes.c_int32(0)
+    with torch.cuda.device(arena.device):
+        st = load().fef_spec_verify_host(
+            draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
+            None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
+            int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
+            out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(), ctypes.byref(status),
+            arena.data_ptr(), arena.numel(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_spec_verify_host")
+    return HostVerifyResult(out.accept_len, out.tokens, out.conf, int(status.value))
+
+
+def fef_remask_select_host_arena_bytes(B: int, L: int, k: int) -> int:
+    return int(load().fef_remask_select_host_arena_bytes(B, L, k))
+
+
+def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena: torch.Tensor,
+                           positions: Optional[torch.Tensor] = None, count: Optional[torch.Tensor] = None,
+                           stream=None):
+    """Host-buffer form of ``fef_remask_select``: CPU tensors in and out, staged through ``arena``."""
+    _require_cuda(arena)
+    if mask.dtype == torch.bool:
+        mask = mask.view(torch.uint8)
+    if conf.device.type != "cpu" or mask.device.type != "cpu" or conf.shape != mask.shape or conf.dim() != 2:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_remask_select_host")
+    B, L = conf.shape
+    if positions is None:
+        positions = torch.empty((B, max(int(k), 0)), dtype=torch.int32).pin_memory()
+    if count is None:
+        count = torch.empty(B, dtype=torch.int32).pin_memory()
+    with torch.cuda.device(arena.device):
+        st = load().fef_remask_select_host(conf.data_ptr(), mask.data_ptr(), B, L, int(k),
+                                           positions.data_ptr() if positions.numel() else None, count.data_ptr(),
+                                           arena.data_ptr(), arena.numel(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_remask_select_host")
+    return positions, count
+
+
+__all__ = ["HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
+           "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]

@@ -56,10 +56,6 @@ __device__ __forceinline__ float lg2_approx(float x) {
     return y;
 }
 
-// 2^(l * c - ref) with c = c_hi + c_lo (c_lo > 0 so that l = -inf stays -inf).
-__device__ __forceinline__ float exp2_scaled(float l, float c_hi, float c_lo, float ref) {
-    return ex2_approx(fmaf(l, c_lo, fmaf(l, c_hi, -ref)));
-}
 
 // Philox4x32-10 (Salmon et al. 2011): returns the four output words.
 __device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key) {
@@ -91,12 +87,22 @@ template <>
 struct Elem<FEF_F32> {
     static constexpr int kBytes = 4;
     static constexpr int kPerVec = 4;
+    static constexpr bool kSplitScale = true;   // c = c_hi + c_lo, two fused multiply-adds
 };
 template <>
 struct Elem<FEF_BF16> {
     static constexpr int kBytes = 2;
     static constexpr int kPerVec = 8;
+    static constexpr bool kSplitScale = false;  // c = c_hi alone (c_lo is 0)
 };
+
+// 2^(l * c - ref).  With the split scale c = c_hi + c_lo and c_lo > 0, so l = -inf stays -inf.
+template <int DT>
+__device__ __forceinline__ float exp2_scaled(float l, float c_hi, float c_lo, float ref) {
+    float x = fmaf(l, c_hi, -ref);
+    if constexpr (Elem<DT>::kSplitScale) x = fmaf(l, c_lo, x);
+    return ex2_approx(x);
+}
 
 template <int DT>
 __device__ __forceinline__ void unpack(const uint4& w, float (&l)[Elem<DT>::kPerVec]) {

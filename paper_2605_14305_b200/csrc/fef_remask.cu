@@ -94,3 +94,38 @@ extern "C" fef_status fef_remask_select(const float* conf, const uint8_t* mask, 
                                                                                      positions, count);
     return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
+
+static size_t remask_up256(size_t n) { return (n + 255) & ~static_cast<size_t>(255); }
+
+extern "C" size_t fef_remask_select_host_arena_bytes(int B, int L, int k) {
+    if (B < 1 || L < 1 || L > FEF_MAX_REMASK_L || k < 0) return 0;
+    const size_t n = static_cast<size_t>(B);
+    return remask_up256(n * L * 4) + remask_up256(n * L) + remask_up256(n * (k > 0 ? k : 1) * 4) + remask_up256(n * 4);
+}
+
+extern "C" fef_status fef_remask_select_host(const float* conf, const uint8_t* mask, int B, int L, int k,
+                                              int32_t* positions, int32_t* count, void* device_arena,
+                                              size_t device_arena_bytes, void* cuda_stream) {
+    if (!conf || !mask || !count || B < 1 || L < 1 || L > FEF_MAX_REMASK_L || k < 0) return FEF_ERR_INVALID_ARG;
+    if (k > 0 && !positions) return FEF_ERR_INVALID_ARG;
+    const size_t need = fef_remask_select_host_arena_bytes(B, L, k);
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255) || device_arena_bytes < need)
+        return FEF_ERR_WORKSPACE;
+    const size_t n = static_cast<size_t>(B);
+    char* d = static_cast<char*>(device_arena);
+    float* d_conf = reinterpret_cast<float*>(d);
+    uint8_t* d_mask = reinterpret_cast<uint8_t*>(d + remask_up256(n * L * 4));
+    int32_t* d_pos = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(d_mask) + remask_up256(n * L));
+    int32_t* d_cnt = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(d_pos) + remask_up256(n * (k > 0 ? k : 1) * 4));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(d_conf, conf, n * L * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(d_mask, mask, n * L, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return FEF_ERR_CUDA;
+    const fef_status st = fef_remask_select(d_conf, d_mask, B, L, k, d_pos, d_cnt, cuda_stream);
+    if (st != FEF_OK) return st;
+    if ((k > 0 && cudaMemcpyAsync(positions, d_pos, n * k * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) ||
+        cudaMemcpyAsync(count, d_cnt, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return FEF_ERR_CUDA;
+    return FEF_OK;
+}

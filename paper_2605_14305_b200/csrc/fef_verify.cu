@@ -83,7 +83,7 @@ __device__ __forceinline__ void absorb_vector(const uint4& w, int first_index, f
     float l[N], e[N];
     unpack<DT>(w, l);
 #pragma unroll
-    for (int i = 0; i < N; ++i) e[i] = exp2_scaled(l[i], c_hi, c_lo, st.ref);
+    for (int i = 0; i < N; ++i) e[i] = exp2_scaled<DT>(l[i], c_hi, c_lo, st.ref);
     float vs;
     if constexpr (N == 8)
         vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
@@ -107,7 +107,7 @@ __device__ __forceinline__ void absorb_vector(const uint4& w, int first_index, f
             st.sum *= ex2_approx(st.ref - nref);
             st.ref = nref;
 #pragma unroll
-            for (int i = 0; i < N; ++i) e[i] = exp2_scaled(l[i], c_hi, c_lo, nref);
+            for (int i = 0; i < N; ++i) e[i] = exp2_scaled<DT>(l[i], c_hi, c_lo, nref);
             if constexpr (N == 8)
                 vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
             else
@@ -130,6 +130,50 @@ __device__ __forceinline__ void absorb_vector(const uint4& w, int first_index, f
             st.best = vmax;
             st.index = first_index + at;
         }
+    }
+}
+
+// Fast path for a full tile (sampling mode): kVecPerThread vectors per thread, packed
+// two-wide binary32 arithmetic (fma.rn.f32x2 / add.f32x2), one overflow check per tile.
+// When the check fires (reference missing or far too low, or bad data) the tile is
+// redone vector by vector through absorb_vector, which moves the reference.
+template <int DT>
+__device__ __forceinline__ void absorb_full_tile(const uint4 (&w)[kVecPerThread], float c_hi, float c_lo,
+                                                 RowState& st) {
+    const float2 ch = make_float2(c_hi, c_hi);
+    const float2 cl = make_float2(c_lo, c_lo);
+    const float2 nref = make_float2(-st.ref, -st.ref);
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        float2 l[4];
+        if constexpr (DT == FEF_F32) {
+            l[0] = make_float2(__uint_as_float(w[j].x), __uint_as_float(w[j].y));
+            l[1] = make_float2(__uint_as_float(w[j].z), __uint_as_float(w[j].w));
+        } else {
+            l[0] = make_float2(__uint_as_float(w[j].x << 16), __uint_as_float(w[j].x & 0xFFFF0000u));
+            l[1] = make_float2(__uint_as_float(w[j].y << 16), __uint_as_float(w[j].y & 0xFFFF0000u));
+            l[2] = make_float2(__uint_as_float(w[j].z << 16), __uint_as_float(w[j].z & 0xFFFF0000u));
+            l[3] = make_float2(__uint_as_float(w[j].w << 16), __uint_as_float(w[j].w & 0xFFFF0000u));
+        }
+#pragma unroll
+        for (int k = 0; k < Elem<DT>::kPerVec / 2; ++k) {
+            float2 x = __ffma2_rn(l[k], ch, nref);
+            if constexpr (Elem<DT>::kSplitScale) x = __ffma2_rn(l[k], cl, x);
+            const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+            if (k & 1)
+                acc1 = __fadd2_rn(acc1, e);
+            else
+                acc0 = __fadd2_rn(acc0, e);
+        }
+    }
+    const float2 acc = __fadd2_rn(acc0, acc1);
+    const float ts = acc.x + acc.y;
+    if (ts <= kRescaleAbove) {
+        st.sum += ts;
+    } else {
+#pragma unroll
+        for (int j = 0; j < kVecPerThread; ++j) absorb_vector<DT, false>(w[j], 0, c_hi, c_lo, st);
     }
 }
 
@@ -263,10 +307,14 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyP
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
                 ++issued;
+                if (!GREEDY && len == kTileBytes) {
+                    absorb_full_tile<DT>(w, P.c_hi, P.c_lo, st);
+                } else {
 #pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j)
-                    if (at[j] < len)
-                        absorb_vector<DT, GREEDY>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+                    for (int j = 0; j < kVecPerThread; ++j)
+                        if (at[j] < len)
+                            absorb_vector<DT, GREEDY>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+                }
             }
             if (++t == G.tiles_per_unit || g + 1 == g_end) {
                 if (have_row) {
@@ -596,7 +644,7 @@ __global__ void __launch_bounds__(kResidualThreads) residual_kernel(const Verify
         unpack<DT>(ld_global_nc_v4(qrow + static_cast<int64_t>(vec) * 16), lq);
 #pragma unroll
         for (int i = 0; i < N; ++i)
-            r[i] = exp2_scaled(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled(lq[i], P.c_hi, P.c_lo, kq);
+            r[i] = exp2_scaled<DT>(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq[i], P.c_hi, P.c_lo, kq);
 #pragma unroll
         for (int g4 = 0; g4 < N / 4; ++g4) {
             const float rmax = fmaxf(fmaxf(r[4 * g4], r[4 * g4 + 1]), fmaxf(r[4 * g4 + 2], r[4 * g4 + 3]));
@@ -617,7 +665,7 @@ __global__ void __launch_bounds__(kResidualThreads) residual_kernel(const Verify
     if (part == 0) {
         for (int x = G.vec_elems + threadIdx.x; x < G.V; x += kResidualThreads) {
             const float lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
-            const float r = exp2_scaled(lp, P.c_hi, P.c_lo, kp) - exp2_scaled(lq, P.c_hi, P.c_lo, kq);
+            const float r = exp2_scaled<DT>(lp, P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq, P.c_hi, P.c_lo, kq);
             if (r > 0.f) {
                 const uint4 w = philox4x32_10(
                     make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), ub, upos, P.step), key);
@@ -790,17 +838,25 @@ static cudaError_t allow_large_smem(Kernel k, int dev, int which, size_t bytes) 
     return e;
 }
 
+static void mark(void* const* events, int which, cudaStream_t stream) {
+    if (events && events[which]) cudaEventRecord(static_cast<cudaEvent_t>(events[which]), stream);
+}
+
 template <int DT, bool GREEDY>
-static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream) {
+static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream, void* const* events) {
     const Geometry& G = P.geo;
     const size_t smem = static_cast<size_t>(kStages) * kTileBytes + 2 * kStages * sizeof(uint64_t) + 16;
+    mark(events, 0, stream);
     if (G.num_tiles > 0) {
         cudaError_t e = allow_large_smem(stream_kernel<DT, GREEDY>, dev, DT * 2 + (GREEDY ? 1 : 0), smem);
         if (e != cudaSuccess) return e;
         stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, smem, stream>>>(P);
     }
+    mark(events, 1, stream);
     scan_kernel<DT, GREEDY><<<G.B, kScanWarps * 32, 0, stream>>>(P);
+    mark(events, 2, stream);
     if (!GREEDY) residual_kernel<DT><<<dim3(G.residual_ctas, G.B), kResidualThreads, 0, stream>>>(P);
+    mark(events, 3, stream);
     return cudaGetLastError();
 }
 
@@ -832,11 +888,12 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
     return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
 }
 
-fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
-                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
-                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
-                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
-                           int32_t* device_status, void* cuda_stream) {
+fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
+                                    int64_t ld, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
+                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
+                                    void* const* stage_events) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -860,13 +917,20 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, 
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return FEF_ERR_WORKSPACE;
 
-    // c = log2(e) / T as c_hi + c_lo with c_lo > 0 (greedy mode reports T = 1 confidences)
+    // c = log2(e) / T (greedy mode reports T = 1 confidences).  binary32 logits: c = c_hi + c_lo
+    // with c_lo > 0, applied with two fused multiply-adds.  bfloat16 logits: the nearest binary32
+    // number alone (c_lo = 0), i.e. the softmax is evaluated at T (1 + d) with |d| <= 6e-8.
     const double c = 1.4426950408889634074 / (greedy ? 1.0 : static_cast<double>(temperature));
     float c_hi = static_cast<float>(c);
-    if (static_cast<double>(c_hi) >= c) c_hi = nextafterf(c_hi, 0.0f);
+    if (dt == FEF_F32) {
+        if (static_cast<double>(c_hi) >= c) c_hi = nextafterf(c_hi, 0.0f);
+        P.c_lo = static_cast<float>(c - static_cast<double>(c_hi));
+        if (!(P.c_lo > 0.f)) return FEF_ERR_INVALID_ARG;
+    } else {
+        P.c_lo = 0.f;
+    }
     P.c_hi = c_hi;
-    P.c_lo = static_cast<float>(c - static_cast<double>(c_hi));
-    if (!(P.c_hi > 0.f) || !(P.c_lo > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
+    if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
 
     P.target = static_cast<const char*>(target_logits);
     P.draft = static_cast<const char*>(draft_logits);
@@ -888,10 +952,103 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, 
         return FEF_ERR_CUDA;
     cudaError_t e;
     if (dt == FEF_F32)
-        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream) : launch_all<FEF_F32, false>(P, dev, stream);
+        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream, stage_events)
+                   : launch_all<FEF_F32, false>(P, dev, stream, stage_events);
     else
-        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream) : launch_all<FEF_BF16, false>(P, dev, stream);
+        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream, stage_events)
+                   : launch_all<FEF_BF16, false>(P, dev, stream, stage_events);
     return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* cuda_stream) {
+    return fef_spec_verify_profiled(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt,
+                                    temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes,
+                                    device_status, cuda_stream, nullptr);
+}
+
+// ---- host-buffer variant: layout of the caller's device arena
+namespace {
+struct ArenaLayout {
+    size_t q, p, tok, row_len, accept_len, tokens, conf, status, workspace, total;
+};
+size_t up256(size_t n) { return (n + 255) & ~static_cast<size_t>(255); }
+bool arena_layout(int B, int K, int V, int64_t ld, fef_dtype dt, ArenaLayout* L) {
+    if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V) return false;
+    if (dt != FEF_F32 && dt != FEF_BF16) return false;
+    const size_t ws = fef_spec_verify_workspace_bytes(B, K, V, dt);
+    if (ws == 0) return false;
+    const size_t logits = static_cast<size_t>(B) * K * ld * (dt == FEF_F32 ? 4 : 2);
+    size_t at = 0;
+    L->q = at; at += up256(logits);
+    L->p = at; at += up256(logits);
+    L->tok = at; at += up256(static_cast<size_t>(B) * K * 4);
+    L->row_len = at; at += up256(static_cast<size_t>(B) * 4);
+    L->accept_len = at; at += up256(static_cast<size_t>(B) * 4);
+    L->tokens = at; at += up256(static_cast<size_t>(B) * K * 4);
+    L->conf = at; at += up256(static_cast<size_t>(B) * K * 4);
+    L->status = at; at += 256;
+    L->workspace = at; at += up256(ws);
+    L->total = at;
+    return true;
+}
+}  // namespace
+
+size_t fef_spec_verify_host_arena_bytes(int B, int K, int V, int64_t ld, fef_dtype dt) {
+    ArenaLayout L;
+    return arena_layout(B, K, V, ld, dt, &L) ? L.total : 0;
+}
+
+fef_status fef_spec_verify_host(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                                const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                                float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                                int32_t* tokens, float* conf, int32_t* status_out, void* device_arena,
+                                size_t device_arena_bytes, void* cuda_stream) {
+    if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
+    if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
+        return FEF_ERR_INVALID_ARG;
+    ArenaLayout L;
+    if (!arena_layout(B, K, V, ld, dt, &L)) {
+        int dev;
+        return cudaGetDevice(&dev) == cudaSuccess ? FEF_ERR_INVALID_ARG : FEF_ERR_CUDA;
+    }
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255) || device_arena_bytes < L.total)
+        return FEF_ERR_WORKSPACE;
+    char* d = static_cast<char*>(device_arena);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t logits = static_cast<size_t>(B) * K * ld * (dt == FEF_F32 ? 4 : 2);
+    const bool greedy = temperature == 0.0f;
+    bool ok = true;
+    if (!greedy) ok = ok && cudaMemcpyAsync(d + L.q, draft_logits, logits, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + L.p, target_logits, logits, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d + L.tok, draft_tokens, static_cast<size_t>(B) * K * 4, cudaMemcpyHostToDevice,
+                               stream) == cudaSuccess;
+    if (row_len)
+        ok = ok && cudaMemcpyAsync(d + L.row_len, row_len, static_cast<size_t>(B) * 4, cudaMemcpyHostToDevice,
+                                   stream) == cudaSuccess;
+    if (!ok) return FEF_ERR_CUDA;
+    const fef_status st = fef_spec_verify(
+        d + L.q, d + L.p, reinterpret_cast<const int32_t*>(d + L.tok),
+        row_len ? reinterpret_cast<const int32_t*>(d + L.row_len) : nullptr, B, K, V, ld, dt, temperature, seed, step,
+        reinterpret_cast<int32_t*>(d + L.accept_len), reinterpret_cast<int32_t*>(d + L.tokens),
+        reinterpret_cast<float*>(d + L.conf), d + L.workspace, device_arena_bytes - L.workspace,
+        reinterpret_cast<int32_t*>(d + L.status), cuda_stream);
+    if (st != FEF_OK) return st;
+    int32_t status_word = 0;
+    ok = ok && cudaMemcpyAsync(accept_len, d + L.accept_len, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost,
+                               stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(tokens, d + L.tokens, static_cast<size_t>(B) * K * 4, cudaMemcpyDeviceToHost,
+                               stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(conf, d + L.conf, static_cast<size_t>(B) * K * 4, cudaMemcpyDeviceToHost, stream) ==
+                   cudaSuccess;
+    ok = ok && cudaMemcpyAsync(&status_word, d + L.status, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    if (!ok) return FEF_ERR_CUDA;
+    if (status_out) *status_out = status_word;
+    return FEF_OK;
 }
 
 }  // extern "C"

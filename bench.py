@@ -212,24 +212,29 @@ def run_native(args):
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
+    # timed region 1: the K steps as a user runs them (kernels chained with dependent launches)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record(stream)
     for i in range(steps):
-        step(warmup + i, stage_ev[i] if not args.no_stage_events else None)
+        step(warmup + i)
     t1.record(stream)
     barrier()
-    sampler.stop()
     elapsed_ms = t0.elapsed_time(t1)
-    status = int(out.device_status.item())
-    accept_mean = float(out.accept_len.float().mean().item())
-    rejected = int((out.accept_len < w.K).sum().item())
-
+    # timed region 2: the same K steps again with CUDA events at the stage boundaries
+    # (fef_spec_verify_profiled), for the per-kernel durations of the roofline
     stage_ms = [0.0, 0.0, 0.0]
     if not args.no_stage_events:
+        for i in range(steps):
+            step(warmup + i, stage_ev[i])
+        barrier()
         for evs in stage_ev:
             for j in range(3):
                 stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
         stage_ms = [x / steps for x in stage_ms]
+    sampler.stop()
+    status = int(out.device_status.item())
+    accept_mean = float(out.accept_len.float().mean().item())
+    rejected = int((out.accept_len < w.K).sum().item())
 
     # ---- end to end through the host-buffer entry points (copies inside the timed region)
     e2e_steps = max(1, min(steps, args.e2e_steps))
@@ -309,6 +314,7 @@ def run_native(args):
         roof["frac"] = roof["achieved"] / peak
         roof["ms_per_launch"] = stage_ms[0]
         roof["stage_ms"] = {"stream": stage_ms[0], "scan": stage_ms[1], "residual": stage_ms[2]}
+        roof["timed"] = "second pass over the same K steps with CUDA events at the kernel boundaries"
     else:
         roof["achieved"], roof["frac"] = None, None
     call_bytes = synth.algorithmic_bytes(w, rejected_rows=rejected)

@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kRemaskThreads) remask_kernel(const float* __r
                                                                int32_t* __restrict__ count) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
+    cudaGridDependencySynchronize();  // conf may come straight from a verification call on this stream
     const int b = blockIdx.x;
     const float* c = conf + static_cast<int64_t>(b) * L;
     const uint8_t* m = mask + static_cast<int64_t>(b) * L;
@@ -90,9 +91,20 @@ extern "C" fef_status fef_remask_select(const float* conf, const uint8_t* mask, 
             return FEF_ERR_CUDA;
         g_remask_attr_done[dev] = true;
     }
-    remask_kernel<<<B, kRemaskThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(conf, mask, L, k, n_sort,
-                                                                                     positions, count);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    // programmatic dependent launch: the grid may be scheduled while the previous kernel on the
+    // stream drains; the kernel waits for it before reading anything
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.blockDim = dim3(kRemaskThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, remask_kernel, conf, mask, L, k, n_sort, positions, count);
+    return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 static size_t remask_up256(size_t n) { return (n + 255) & ~static_cast<size_t>(255); }

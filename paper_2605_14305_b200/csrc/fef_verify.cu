@@ -133,47 +133,68 @@ __device__ __forceinline__ void absorb_vector(const uint4& w, int first_index, f
     }
 }
 
-// Fast path for a full tile (sampling mode): kVecPerThread vectors per thread, packed
-// two-wide binary32 arithmetic (fma.rn.f32x2 / add.f32x2), one overflow check per tile.
-// When the check fires (reference missing or far too low, or bad data) the tile is
-// redone vector by vector through absorb_vector, which moves the reference.
+// One 16-byte vector, packed two-wide binary32 arithmetic (fma.rn.f32x2 / add.f32x2):
+// adds 2^(l*c - ref) of its elements to two running pair-sums.  No overflow check here.
 template <int DT>
-__device__ __forceinline__ void absorb_full_tile(const uint4 (&w)[kVecPerThread], float c_hi, float c_lo,
-                                                 RowState& st) {
+__device__ __forceinline__ void add_vector_packed(const uint4& w, float2 ch, float2 cl, float2 nref,
+                                                  float2& acc0, float2& acc1) {
+    float2 l[4];
+    if constexpr (DT == FEF_F32) {
+        l[0] = make_float2(__uint_as_float(w.x), __uint_as_float(w.y));
+        l[1] = make_float2(__uint_as_float(w.z), __uint_as_float(w.w));
+    } else {
+        l[0] = make_float2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
+        l[1] = make_float2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+        l[2] = make_float2(__uint_as_float(w.z << 16), __uint_as_float(w.z & 0xFFFF0000u));
+        l[3] = make_float2(__uint_as_float(w.w << 16), __uint_as_float(w.w & 0xFFFF0000u));
+    }
+#pragma unroll
+    for (int k = 0; k < Elem<DT>::kPerVec / 2; ++k) {
+        float2 x = __ffma2_rn(l[k], ch, nref);
+        if constexpr (Elem<DT>::kSplitScale) x = __ffma2_rn(l[k], cl, x);
+        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+        if (k & 1)
+            acc1 = __fadd2_rn(acc1, e);
+        else
+            acc0 = __fadd2_rn(acc0, e);
+    }
+}
+
+// Reference exponent for a row that has none yet: c * (largest element of the thread's
+// first vector), or "none" when that vector holds no finite number.
+template <int DT>
+__device__ __forceinline__ float first_reference(const uint4& w, float c_hi, float c_lo) {
+    constexpr int N = Elem<DT>::kPerVec;
+    float l[N];
+    unpack<DT>(w, l);
+    float vmax = l[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, l[i]);
+    return (vmax > -INFINITY && vmax < INFINITY) ? fmaf(vmax, c_lo, vmax * c_hi) : kNoReference;
+}
+
+// A thread's share of one tile in sampling mode: the vectors with offset < len, one
+// overflow check for the whole tile.  When the check fires (reference far too low or
+// missing, or bad data) the tile is redone vector by vector through absorb_vector,
+// which moves the reference.
+template <int DT, bool FULL>
+__device__ __forceinline__ void absorb_tile(const uint4 (&w)[kVecPerThread], const int (&at)[kVecPerThread], int len,
+                                            float c_hi, float c_lo, RowState& st) {
     const float2 ch = make_float2(c_hi, c_hi);
     const float2 cl = make_float2(c_lo, c_lo);
     const float2 nref = make_float2(-st.ref, -st.ref);
     float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < kVecPerThread; ++j) {
-        float2 l[4];
-        if constexpr (DT == FEF_F32) {
-            l[0] = make_float2(__uint_as_float(w[j].x), __uint_as_float(w[j].y));
-            l[1] = make_float2(__uint_as_float(w[j].z), __uint_as_float(w[j].w));
-        } else {
-            l[0] = make_float2(__uint_as_float(w[j].x << 16), __uint_as_float(w[j].x & 0xFFFF0000u));
-            l[1] = make_float2(__uint_as_float(w[j].y << 16), __uint_as_float(w[j].y & 0xFFFF0000u));
-            l[2] = make_float2(__uint_as_float(w[j].z << 16), __uint_as_float(w[j].z & 0xFFFF0000u));
-            l[3] = make_float2(__uint_as_float(w[j].w << 16), __uint_as_float(w[j].w & 0xFFFF0000u));
-        }
-#pragma unroll
-        for (int k = 0; k < Elem<DT>::kPerVec / 2; ++k) {
-            float2 x = __ffma2_rn(l[k], ch, nref);
-            if constexpr (Elem<DT>::kSplitScale) x = __ffma2_rn(l[k], cl, x);
-            const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-            if (k & 1)
-                acc1 = __fadd2_rn(acc1, e);
-            else
-                acc0 = __fadd2_rn(acc0, e);
-        }
-    }
+    for (int j = 0; j < kVecPerThread; ++j)
+        if (FULL || at[j] < len) add_vector_packed<DT>(w[j], ch, cl, nref, acc0, acc1);
     const float2 acc = __fadd2_rn(acc0, acc1);
     const float ts = acc.x + acc.y;
     if (ts <= kRescaleAbove) {
         st.sum += ts;
     } else {
 #pragma unroll
-        for (int j = 0; j < kVecPerThread; ++j) absorb_vector<DT, false>(w[j], 0, c_hi, c_lo, st);
+        for (int j = 0; j < kVecPerThread; ++j)
+            if (FULL || at[j] < len) absorb_vector<DT, false>(w[j], 0, c_hi, c_lo, st);
     }
 }
 
@@ -307,13 +328,17 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyP
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
                 ++issued;
-                if (!GREEDY && len == kTileBytes) {
-                    absorb_full_tile<DT>(w, P.c_hi, P.c_lo, st);
-                } else {
+                if constexpr (GREEDY) {
 #pragma unroll
                     for (int j = 0; j < kVecPerThread; ++j)
                         if (at[j] < len)
-                            absorb_vector<DT, GREEDY>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+                            absorb_vector<DT, true>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+                } else {
+                    if (st.ref == kNoReference && at[0] < len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
+                    if (len == kTileBytes)  // branch-free: the four vectors interleave
+                        absorb_tile<DT, true>(w, at, len, P.c_hi, P.c_lo, st);
+                    else
+                        absorb_tile<DT, false>(w, at, len, P.c_hi, P.c_lo, st);
                 }
             }
             if (++t == G.tiles_per_unit || g + 1 == g_end) {
@@ -380,14 +405,23 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
     const Partial* rec = P.partials + u * G.max_slots * kConsumerWarps;
     const int ntail = G.V - G.vec_elems;
 
-    double M = -INFINITY;
+    // each lane folds its records into a running (m, s) pair, then the warp combines
+    double m = -INFINITY, sacc = 0.0;
     int bad = 0;
     float best = -INFINITY;
     int index = 0x7FFFFFFF;
     for (int r = lane; r < nrec; r += 32) {
         const Partial p = rec[r];
         if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = 1;
-        if (p.sum > 0.f) M = fmax(M, static_cast<double>(p.ref));
+        if (p.sum > 0.f) {
+            const double pm = p.ref, ps = p.sum;
+            if (pm > m) {
+                sacc = sacc * exp2(m - pm) + ps;
+                m = pm;
+            } else {
+                sacc += ps * exp2(pm - m);
+            }
+        }
         if (GREEDY && better(p.best, p.index, best, index)) {
             best = p.best;
             index = p.index;
@@ -395,14 +429,23 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
     }
     for (int j = lane; j < ntail; j += 32) {
         const float l = load_logit<DT>(row, G.vec_elems + j);
-        if (l != l || l == INFINITY) bad = 1;
-        else if (l > -INFINITY) M = fmax(M, static_cast<double>(l) * c);
+        if (l != l || l == INFINITY) {
+            bad = 1;
+        } else if (l > -INFINITY) {
+            const double pm = static_cast<double>(l) * c;
+            if (pm > m) {
+                sacc = sacc * exp2(m - pm) + 1.0;
+                m = pm;
+            } else {
+                sacc += exp2(pm - m);
+            }
+        }
         if (GREEDY && better(l, G.vec_elems + j, best, index)) {
             best = l;
             index = G.vec_elems + j;
         }
     }
-    M = warp_max(M);
+    const double M = warp_max(m);
     bad = __any_sync(0xFFFFFFFFu, bad);
     if (GREEDY) {
 #pragma unroll
@@ -415,19 +458,7 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
             }
         }
     }
-
-    double S = 0.0;
-    if (!bad) {
-        for (int r = lane; r < nrec; r += 32) {
-            const Partial p = rec[r];
-            if (p.sum > 0.f) S += static_cast<double>(p.sum) * exp2(static_cast<double>(p.ref) - M);
-        }
-        for (int j = lane; j < ntail; j += 32) {
-            const float l = load_logit<DT>(row, G.vec_elems + j);
-            if (l > -INFINITY) S += exp2(static_cast<double>(l) * c - M);
-        }
-        S = warp_sum(S);
-    }
+    const double S = warp_sum(m > -INFINITY ? sacc * exp2(m - M) : 0.0);
     RowNorm out;
     out.M = M;
     out.S = S;
@@ -437,11 +468,13 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
     return out;
 }
 
-constexpr int kScanWarps = 8;
+constexpr int kScanMaxWarps = 32;
 
 template <int DT, bool GREEDY>
-__global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kScanMaxWarps * 32) scan_kernel(const VerifyParams P) {
     const Geometry& G = P.geo;
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+    const int num_warps = blockDim.x >> 5;
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
@@ -451,7 +484,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const VerifyParam
     __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
     __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
 
-    for (int i = warp; i < n; i += kScanWarps) {
+    for (int i = warp; i < n; i += num_warps) {
         const int64_t row = static_cast<int64_t>(b) * G.K + i;
         const char* prow = P.target + row * G.ld_bytes;
         const char* qrow = P.draft + row * G.ld_bytes;
@@ -508,8 +541,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const VerifyParam
     for (int i = n - 1; i >= 0; --i)
         if (!s_accept[i]) a = i;
 
-    const int i = threadIdx.x;
-    if (i < G.K) {
+    for (int i = threadIdx.x; i < G.K; i += blockDim.x) {
         const int64_t row = static_cast<int64_t>(b) * G.K + i;
         int tok = -1;
         float cf = -1.f;
@@ -617,9 +649,10 @@ __device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kResidualThreads) residual_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const VerifyParams P) {
     constexpr int N = Elem<DT>::kPerVec;
     const Geometry& G = P.geo;
+    cudaGridDependencySynchronize();  // the scan kernel's tasks must be complete and visible
     const int b = blockIdx.y, part = blockIdx.x, parts = gridDim.x;
     const ResidualTask task = P.tasks[b];
     if (task.pos < 0) return;  // uniform over the CTA
@@ -806,7 +839,7 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool gr
     if (G.grid < 1) G.grid = 1;
     const int64_t min_tiles_per_cta = G.num_tiles > 0 ? G.num_tiles / G.grid : 1;
     G.max_slots = G.tiles_per_unit > 0 ? static_cast<int>((G.tiles_per_unit - 1) / min_tiles_per_cta) + 2 : 1;
-    int parts = (2 * sm_count + B - 1) / B;
+    int parts = (6 * sm_count + B - 1) / B;
     const int nvec = G.vec_bytes / 16;
     const int max_parts_by_size = nvec / kResidualThreads > 0 ? nvec / kResidualThreads : 1;
     if (parts > max_parts_by_size) parts = max_parts_by_size;
@@ -842,10 +875,30 @@ static void mark(void* const* events, int which, cudaStream_t stream) {
     if (events && events[which]) cudaEventRecord(static_cast<cudaEvent_t>(events[which]), stream);
 }
 
+// Launch with programmatic dependent launch: the grid may be scheduled while its
+// predecessor on the stream drains; the kernel itself waits (cudaGridDependencySynchronize)
+// before touching anything the predecessor wrote.
+template <typename... Args>
+static cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <int DT, bool GREEDY>
 static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream, void* const* events) {
     const Geometry& G = P.geo;
     const size_t smem = static_cast<size_t>(kStages) * kTileBytes + 2 * kStages * sizeof(uint64_t) + 16;
+    const bool timed = events != nullptr;  // event records between kernels rule out dependent launches
     mark(events, 0, stream);
     if (G.num_tiles > 0) {
         cudaError_t e = allow_large_smem(stream_kernel<DT, GREEDY>, dev, DT * 2 + (GREEDY ? 1 : 0), smem);
@@ -853,9 +906,21 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, smem, stream>>>(P);
     }
     mark(events, 1, stream);
-    scan_kernel<DT, GREEDY><<<G.B, kScanWarps * 32, 0, stream>>>(P);
+    const int scan_threads = 32 * (G.K < kScanMaxWarps ? G.K : kScanMaxWarps);
+    cudaError_t e;
+    if (timed)
+        scan_kernel<DT, GREEDY><<<G.B, scan_threads, 0, stream>>>(P), e = cudaGetLastError();
+    else
+        e = launch_dependent(scan_kernel<DT, GREEDY>, dim3(G.B), dim3(scan_threads), 0, stream, P);
+    if (e != cudaSuccess) return e;
     mark(events, 2, stream);
-    if (!GREEDY) residual_kernel<DT><<<dim3(G.residual_ctas, G.B), kResidualThreads, 0, stream>>>(P);
+    if (!GREEDY) {
+        if (timed)
+            residual_kernel<DT><<<dim3(G.residual_ctas, G.B), kResidualThreads, 0, stream>>>(P), e = cudaGetLastError();
+        else
+            e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
+        if (e != cudaSuccess) return e;
+    }
     mark(events, 3, stream);
     return cudaGetLastError();
 }

@@ -38,7 +38,8 @@ typedef enum {
     FEF_ERR_CUDA = 5,        /* CUDA runtime error (see cudaGetLastError), or no device   */
     FEF_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out            */
     FEF_ERR_NONFINITE = 7,   /* device: NaN or +inf logit, or a row that is all -inf      */
-    FEF_ERR_TOKEN_RANGE = 8  /* device: a draft token outside [0, V)                      */
+    FEF_ERR_TOKEN_RANGE = 8, /* device: a draft token outside [0, V)                      */
+    FEF_ERR_TOO_LARGE = 9    /* fef_spec_verify_static: sizes exceed its built-in scratch  */
 } fef_status;
 
 typedef enum { FEF_F32 = 0, FEF_BF16 = 1 } fef_dtype;
@@ -147,6 +148,41 @@ fef_status fef_spec_verify_host(const void* draft_logits, const void* target_log
                                 int32_t* accept_len, int32_t* tokens, float* conf,
                                 int32_t* status_out,
                                 void* device_arena, size_t device_arena_bytes, void* cuda_stream);
+
+/*
+ * fef_spec_verify for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same results.)
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they verify:
+ * code running inside someone else's memory plan (an inference server that hands out
+ * all device memory up front and forbids later allocations), plug-ins that receive
+ * only input and output buffers, and code on a latency path where an allocation -
+ * which may synchronise the device - is not acceptable.  For them the scratch that
+ * fef_spec_verify takes as `workspace` lives inside the library instead: a fixed
+ * device array of FEF_STATIC_SCRATCH_BYTES that every GPU using the library holds from
+ * the moment the library is loaded there until the process exits.  The call itself
+ * allocates and frees nothing.
+ *
+ * Arguments are those of fef_spec_verify without workspace / workspace_bytes; the
+ * caller still owns all inputs and outputs.
+ *   - Sizes whose scratch need (fef_spec_verify_workspace_bytes) exceeds
+ *     FEF_STATIC_SCRATCH_BYTES are refused with FEF_ERR_TOO_LARGE and nothing is
+ *     launched.  The headline shape B = 64, K = 32, V = 126464 needs about 2.3 MB.
+ *   - The first call on each device looks up the array's device address (one runtime
+ *     query, no allocation).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call
+ *     left; no call depends on that content.  Two calls whose kernels can overlap on
+ *     the GPU (different streams, no ordering between them) race on it and give
+ *     undefined results: keep calls of this entry point ordered, or use fef_spec_verify
+ *     with separate workspaces.
+ */
+#define FEF_STATIC_SCRATCH_BYTES (8u << 20)
+fef_status fef_spec_verify_static(const void* draft_logits, const void* target_logits,
+                                  const int32_t* draft_tokens, const int32_t* row_len,
+                                  int B, int K, int V, int64_t ld, fef_dtype dt,
+                                  float temperature, uint64_t seed, uint32_t step,
+                                  int32_t* accept_len, int32_t* tokens, float* conf,
+                                  int32_t* device_status, void* cuda_stream);
 
 /*
  * LowConf_k of Algorithm 2 ("Select R = LowConf_{n_rm}(C)"): for every batch

@@ -17,13 +17,14 @@ import torch
 from . import _build
 
 FEF_OK, FEF_ERR_INVALID_ARG, FEF_ERR_DTYPE, FEF_ERR_ALIGNMENT, FEF_ERR_WORKSPACE = 0, 1, 2, 3, 4
-FEF_ERR_CUDA, FEF_ERR_TIMEOUT, FEF_ERR_NONFINITE, FEF_ERR_TOKEN_RANGE = 5, 6, 7, 8
+FEF_ERR_CUDA, FEF_ERR_TIMEOUT, FEF_ERR_NONFINITE, FEF_ERR_TOKEN_RANGE, FEF_ERR_TOO_LARGE = 5, 6, 7, 8, 9
+FEF_STATIC_SCRATCH_BYTES = 8 << 20
 FEF_F32, FEF_BF16 = 0, 1
 FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
 
 EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_spec_verify_profiled",
            "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
-           "fef_remask_select_host_arena_bytes", "fef_remask_select_host")
+           "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static")
 
 _lib = None
 
@@ -61,6 +62,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_host_arena_bytes.restype = sz
     L.fef_spec_verify_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp, sz, vp]
     L.fef_spec_verify_host.restype = i32
+    L.fef_spec_verify_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp]
+    L.fef_spec_verify_static.restype = i32
     L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.fef_remask_select.restype = i32
     L.fef_remask_select_host_arena_bytes.argtypes = [i32, i32, i32]
@@ -187,6 +190,42 @@ def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions:
     return positions, count
 
 
+def fef_spec_verify_static(draft_logits: torch.Tensor, target_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                           temperature: float, seed: int, step: int, row_len: Optional[torch.Tensor] = None,
+                           V: Optional[int] = None, out: Optional[VerifyResult] = None, stream=None) -> VerifyResult:
+    """``fef_spec_verify`` without a workspace argument, for callers that must not allocate
+    device memory: the scratch is a fixed array inside the library (see
+    ``fef_spec_verify_static`` in include/fef.h for the size limit, the first-call set-up
+    and the rule that calls sharing a device must not overlap).  ``out`` must be given if
+    the caller wants no allocation at all; without it this wrapper allocates the outputs."""
+    _require_cuda(draft_logits, target_logits, draft_tokens, row_len)
+    if draft_logits.dim() != 3 or draft_logits.shape != target_logits.shape or draft_logits.dtype != target_logits.dtype:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_static")
+    if not (draft_logits.is_contiguous() and target_logits.is_contiguous() and draft_tokens.is_contiguous()):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_static")
+    if draft_tokens.dtype != torch.int32 or (row_len is not None and row_len.dtype != torch.int32):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_static")
+    B, K, ld = draft_logits.shape
+    V = ld if V is None else int(V)
+    code = _dtype_code(draft_logits)
+    dev = draft_logits.device
+    with torch.cuda.device(dev):
+        if out is None:
+            out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.float32, device=dev),
+                               torch.empty(1, dtype=torch.int32, device=dev))
+        st = load().fef_spec_verify_static(
+            draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
+            None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
+            int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
+            out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
+            out.device_status.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_spec_verify_static")
+    return out
+
+
 def fef_spec_verify_host_arena_bytes(B: int, K: int, V: int, ld: int, dtype) -> int:
     code = dtype if isinstance(dtype, int) else (FEF_F32 if dtype == torch.float32 else FEF_BF16)
     return int(load().fef_spec_verify_host_arena_bytes(B, K, V, ld, code))
@@ -257,6 +296,6 @@ def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena
     return positions, count
 
 
-__all__ = ["HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
+__all__ = ["fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]

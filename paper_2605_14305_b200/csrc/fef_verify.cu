@@ -940,6 +940,7 @@ const char* fef_status_string(fef_status s) {
         case FEF_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         case FEF_ERR_NONFINITE: return "NaN or +inf logit, or a row of -inf only";
         case FEF_ERR_TOKEN_RANGE: return "draft token outside [0, V)";
+        case FEF_ERR_TOO_LARGE: return "sizes need more scratch than the built-in buffer of fef_spec_verify_static holds";
     }
     return "unknown status";
 }
@@ -1114,6 +1115,40 @@ fef_status fef_spec_verify_host(const void* draft_logits, const void* target_log
     if (!ok) return FEF_ERR_CUDA;
     if (status_out) *status_out = status_word;
     return FEF_OK;
+}
+
+// ---- variant for callers that cannot allocate device memory
+//
+// Scratch for fef_spec_verify_static.  It is part of the library image: every GPU that loads
+// the library carries these FEF_STATIC_SCRATCH_BYTES until the process exits.  In host code
+// the name below is only a handle for the runtime (not a device address); the address the
+// kernels get comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[FEF_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_address[64];  // per device, filled on the first call there
+
+fef_status fef_spec_verify_static(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                                  const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                                  float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                                  int32_t* tokens, float* conf, int32_t* device_status, void* cuda_stream) {
+    if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
+    if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V) return FEF_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FEF_ERR_CUDA;
+    const size_t need = fef_spec_verify_workspace_bytes(B, K, V, dt);
+    if (need == 0) return FEF_ERR_INVALID_ARG;
+    if (need > FEF_STATIC_SCRATCH_BYTES) return FEF_ERR_TOO_LARGE;
+    void* scratch = g_static_scratch_address[dev];
+    if (!scratch) {
+        // set-up, once per device, with that device current: ask the runtime where the array lives
+        if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return FEF_ERR_CUDA;
+        g_static_scratch_address[dev] = scratch;
+    }
+    // Nothing in the scratch has to start at zero: the streaming kernel overwrites every partial
+    // the scan reads, and the scan rewrites every window's task (arrival counter included)
+    // before the residual kernel looks at it, so leftovers of earlier calls are never read.
+    return fef_spec_verify(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt, temperature, seed,
+                           step, accept_len, tokens, conf, scratch, FEF_STATIC_SCRATCH_BYTES, device_status,
+                           cuda_stream);
 }
 
 }  // extern "C"

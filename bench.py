@@ -163,6 +163,7 @@ def run_native(args):
     import torch.distributed as dist
 
     import paper_2605_14305_b200 as fef
+    from paper_2605_14305_b200 import dist_util
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -178,6 +179,7 @@ def run_native(args):
     w = _workload(args)
     steps, warmup = args.steps, max(args.warmup, 3)
     nbuf = 2
+    seed = dist_util.rank_seed(args.seed, rank)
     sets = [synth.make_call(w, seed=1000 * (rank + 1) + i, device=dev) for i in range(nbuf)]
     g = torch.Generator(device=dev).manual_seed(77 + rank)
     conf_state = torch.rand((w.B, REMASK_L), generator=g, device=dev)
@@ -199,7 +201,7 @@ def run_native(args):
 
     def step(i, events=None):
         q, p, tok = sets[i % nbuf]
-        fef.fef_spec_verify(q, p, tok, w.temperature, args.seed, i, out=out, workspace=ws, stage_events=events)
+        fef.fef_spec_verify(q, p, tok, w.temperature, seed, i, out=out, workspace=ws, stage_events=events)
         fef.fef_remask_select(conf_state, mask_state, w.remask_k, positions=positions, count=count)
 
     def barrier():
@@ -249,7 +251,7 @@ def run_native(args):
     hcnt = torch.empty(w.B, dtype=torch.int32).pin_memory()
 
     def host_step(i):
-        fef.fef_spec_verify_host(hq, hp, htok, w.temperature, args.seed, i, arena, out=hout)
+        fef.fef_spec_verify_host(hq, hp, htok, w.temperature, seed, i, arena, out=hout)
         fef.fef_remask_select_host(hconf, hmask, w.remask_k, arena2, positions=hpos, count=hcnt)
 
     host_step(0)
@@ -262,10 +264,7 @@ def run_native(args):
     barrier()
     e2e_ms = h0.elapsed_time(h1)
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    elapsed_ms, e2e_ms = dist_util.max_over_ranks([elapsed_ms, e2e_ms], device=dev)
 
     logits_bytes = hq.numel() * hq.element_size() * (2 if w.temperature > 0 else 1)
     h2d = logits_bytes + htok.numel() * 4 + hconf.numel() * 4 + hmask.numel()
@@ -303,7 +302,7 @@ def run_native(args):
         return
 
     positions_per_step = w.B * w.K * world
-    value = positions_per_step * steps / (elapsed_ms * 1e-3)
+    value = dist_util.aggregate_rate(w.B * w.K, steps, elapsed_ms, world)
     peak, peak_src = _measured_peak()
     row_bytes = (2 if w.temperature > 0 else 1) * w.V * w.logit_bytes
     stream_bytes = w.B * w.K * row_bytes

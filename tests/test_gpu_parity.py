@@ -297,3 +297,68 @@ def test_remask_select_nan_sorts_last(fef):
     pos, cnt = fef.fef_remask_select(conf, mask, 6)
     opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), 6)
     assert pos.cpu().numpy().tolist() == opos.tolist() == [[5, 2, 0, 3, 1, 4]]
+
+
+def test_host_buffer_entry_points_match_device_entry_points(fef):
+    """fef_spec_verify_host / fef_remask_select_host: same results from pinned and from pageable host memory."""
+    q, p, tok = _random_case(6, 8, 20000, torch.bfloat16, 0.7, 41)
+    row_len = torch.tensor([8, 8, 3, 0, 8, 5], dtype=torch.int32, device="cuda")
+    want = _gpu_verify(fef, q, p, tok, 0.9, 12, 13, row_len=row_len)
+    arena = torch.empty(fef.fef_spec_verify_host_arena_bytes(6, 8, 20000, 20000, torch.bfloat16), dtype=torch.uint8,
+                        device="cuda")
+    for pin in (True, False):
+        hq, hp, htok, hrl = (t.cpu().pin_memory() if pin else t.cpu() for t in (q, p, tok, row_len))
+        got = fef.fef_spec_verify_host(hq, hp, htok, 0.9, 12, 13, arena, row_len=hrl)
+        assert got.status == 0
+        assert (got.accept_len.numpy() == want[0]).all() and (got.tokens.numpy() == want[1]).all()
+        assert (got.conf.numpy() == want[2]).all()
+    got = fef.fef_spec_verify_host(hq, hp, htok, 0.0, 12, 14, arena)
+    want = _gpu_verify(fef, q, p, tok, 0.0, 12, 14)
+    assert (got.tokens.numpy() == want[1]).all()
+    conf = torch.rand(4, 300)
+    mask = (torch.rand(4, 300) < 0.5).to(torch.uint8)
+    arena2 = torch.empty(fef.fef_remask_select_host_arena_bytes(4, 300, 9), dtype=torch.uint8, device="cuda")
+    pos, cnt = fef.fef_remask_select_host(conf, mask, 9, arena2)
+    opos, ocnt = oracle.remask_select(conf, mask, 9)
+    assert (pos.numpy() == opos).all() and (cnt.numpy() == ocnt).all()
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(fef.FefError) as err:
+        fef.fef_spec_verify_host(hq, hp, htok, 0.9, 12, 13, small)
+    assert err.value.status == fef.FEF_ERR_WORKSPACE
+
+
+def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef):
+    q, p, tok = _random_case(4, 16, 50000, torch.bfloat16, 0.7, 51)
+    want = _gpu_verify(fef, q, p, tok, 1.0, 3, 3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for e in ev:
+        e.record()
+    r = fef.fef_spec_verify(q, p, tok, 1.0, 3, 3, stage_events=ev)
+    torch.cuda.synchronize()
+    assert (r.accept_len.cpu().numpy() == want[0]).all() and (r.tokens.cpu().numpy() == want[1]).all()
+    assert (r.conf.cpu().numpy() == want[2]).all()
+    assert all(ev[i].elapsed_time(ev[i + 1]) > 0 for i in range(3))
+
+
+def test_api_errors_with_real_buffers(fef):
+    q, p, tok = _random_case(2, 4, 64, torch.float32, 0.5, 61)
+    lib = fef.load()
+    out = fef.fef_spec_verify(q, p, tok, 1.0, 0, 0)
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+
+    def call(qq=q, V=64, ld=64, K=4, T=1.0, wsb=ws.numel(), wsp=None, dt=0):
+        return lib.fef_spec_verify(qq.data_ptr(), p.data_ptr(), tok.data_ptr(), None, 2, K, V, ld, dt, T, 1, 1,
+                                   out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
+                                   ws.data_ptr() if wsp is None else wsp, wsb, out.device_status.data_ptr(), None)
+    assert call() == fef.FEF_OK
+    assert call(wsb=16) == fef.FEF_ERR_WORKSPACE
+    assert call(wsp=ws.data_ptr() + 8) == fef.FEF_ERR_WORKSPACE
+    assert call(ld=32) == fef.FEF_ERR_INVALID_ARG
+    assert call(K=65) == fef.FEF_ERR_INVALID_ARG
+    assert call(T=-1.0) == fef.FEF_ERR_INVALID_ARG
+    assert call(dt=5) == fef.FEF_ERR_DTYPE
+    assert call(qq=q.view(-1)[1:]) == fef.FEF_ERR_ALIGNMENT
+    assert call(V=10, ld=10) == fef.FEF_ERR_ALIGNMENT
+    torch.cuda.synchronize()
+    assert fef.fef_spec_verify_workspace_bytes(2, 4, 64, torch.float32) > 0
+    assert fef.fef_spec_verify_workspace_bytes(2, 65, 64, torch.float32) == 0

@@ -11,8 +11,9 @@
  * Conventions
  *  - Pointers marked "device" must be device memory of the current CUDA device;
  *    the caller owns every buffer.  The library allocates nothing, keeps no
- *    state between calls and never synchronises: all work is enqueued on
- *    `cuda_stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *    state between calls and never synchronises: all work (one kernel per call,
+ *    preceded by the clearing of a few counters) is enqueued on `cuda_stream`
+ *    (a cudaStream_t passed as void*; NULL = the default stream).
  *  - The return value reports what the host can see (bad arguments, launch
  *    failures).  Errors that only the data reveals are written to
  *    `*device_status` by the kernels; nothing ever traps.
@@ -56,7 +57,9 @@ const char* fef_status_string(fef_status s);
  * Bytes of device scratch fef_spec_verify needs for these sizes on the current
  * CUDA device (it depends on the device's SM count).  Returns 0 for invalid
  * sizes or when no device is available.  The scratch must be 256-byte aligned;
- * its contents need not be initialised and are meaningless afterwards.
+ * its contents need not be initialised (the call clears the counters it keeps
+ * there) and are meaningless afterwards.  Two calls that may overlap on the GPU
+ * need separate scratch buffers.
  */
 size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt);
 
@@ -110,23 +113,6 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
                            int32_t* accept_len, int32_t* tokens, float* conf,
                            void* workspace, size_t workspace_bytes,
                            int32_t* device_status, void* cuda_stream);
-
-/*
- * fef_spec_verify with timing marks: the same operation (Algorithm 2's verification
- * loop), and additionally records up to four caller-created CUDA events
- * (cudaEvent_t passed as void*; NULL entries are skipped) on `cuda_stream`:
- * [0] before the streaming pass, [1] after it, [2] after the acceptance scan,
- * [3] after the residual pass.  `stage_events` may be NULL.  Used to time the
- * stages separately; results are identical to fef_spec_verify.
- */
-fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
-                                    const int32_t* draft_tokens, const int32_t* row_len,
-                                    int B, int K, int V, int64_t ld, fef_dtype dt,
-                                    float temperature, uint64_t seed, uint32_t step,
-                                    int32_t* accept_len, int32_t* tokens, float* conf,
-                                    void* workspace, size_t workspace_bytes,
-                                    int32_t* device_status, void* cuda_stream,
-                                    void* const* stage_events);
 
 /*
  * Host-buffer form of fef_spec_verify (same operation, same citations): every

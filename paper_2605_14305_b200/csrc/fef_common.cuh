@@ -10,18 +10,20 @@ namespace fef {
 
 // ------------------------------------------------------------------ sizes ----
 constexpr int kConsumerWarps = 16;                      // warps that do arithmetic in the streaming kernel
-constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kProducerWarp = kConsumerWarps;           // one thread of it feeds the ring
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
 constexpr int kVecPerThread = 4;                        // 16-byte vectors per thread per tile
 constexpr int kTileBytes = kConsumerWarps * 32 * 16 * kVecPerThread;  // 32 KiB
 constexpr int kStages = 5;                              // ring depth: 160 KiB in flight per SM
 constexpr int kSpinLimit = 1 << 22;                     // bound on every mbarrier wait loop
+constexpr int kSlotSets = 8;                            // in-CTA combine buffers (a warp leads by < 8 flushes)
 
 constexpr float kNoReference = -3.0e38f;                // "no reference yet" for the running softmax
 constexpr float kRescaleAbove = 1.152921504606847e18f;  // 2^60: a vector sum above this re-references
 
-// One partial result of the streaming kernel: a warp's share of one row.
+// One partial result of the streaming kernel: one claim's share of one row.
 //   ref    reference exponent (log2 domain) the sum is relative to
-//   sum    sum_v 2^(l_v * c - ref) over the warp's elements (NaN when the data is bad)
+//   sum    sum_v 2^(l_v * c - ref) over the claim's elements (NaN when the data is bad)
 //   best   largest logit seen (greedy mode only)
 //   index  vocabulary id of `best`, lowest on ties (greedy mode only)
 struct __align__(16) Partial {
@@ -37,6 +39,11 @@ struct __align__(16) ResidualTask {
     unsigned arrivals;  // CTAs of the residual kernel that have finished this window
     double kp;          // log2 normaliser of the target law at a: pi(x) = 2^(l_x * c - kp)
     double kq;          // same for the draft law
+};
+
+// Counter shared by all CTAs of the streaming kernel (cleared by the host call).
+struct __align__(16) Control {
+    unsigned long long next_claim;  // next streaming claim to hand out
 };
 
 struct __align__(8) Candidate {

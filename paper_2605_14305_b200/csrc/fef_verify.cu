@@ -1,15 +1,18 @@
 // fef_spec_verify: the verification loop of the paper's Algorithm 2 for B windows at once.
 //
-// Three kernels, enqueued back to back on the caller's stream:
+// Three kernels, enqueued back to back on the caller's stream (the second and third with
+// programmatic dependent launch):
 //   stream_kernel    reads every target and draft row exactly once (bulk-async copies into a
-//                    shared-memory ring) and leaves, per row, partial sums of
+//                    shared-memory ring; persistent CTAs take runs of tiles, "claims", from a
+//                    shared counter in row order) and leaves, per claim, the partial sum of
 //                    2^(l_v * c - ref), c = log2(e) / T, from which pi(x) and rho(x) follow
 //                    for any x  (the two softmax laws of Section 3.2);
-//   scan_kernel      per window: finishes the normalisers in double precision, draws u_i,
-//                    applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)}, finds the first rejection,
-//                    writes accepted tokens and confidences c_i = pi_i(x_i);
-//   residual_kernel  only for windows that rejected: Gumbel-max draw from
-//                    [pi - rho]_+ over the rejected row, then c = pi(Z).
+//   scan_kernel      one warp per window, one lane per position: finishes the normalisers in
+//                    double precision, draws u_i, applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)},
+//                    finds the first rejection, writes accepted tokens and confidences
+//                    c_i = pi_i(x_i);
+//   residual_kernel  only for windows that rejected: Gumbel-max draw from [pi - rho]_+ over the
+//                    rejected row (the residual law defined before Algorithm 2), then c = pi(Z).
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -23,22 +26,18 @@ namespace fef {
 struct Geometry {
     int B, K, V;
     int units_per_row;    // 2: target row and draft row; 1 in greedy mode (target only)
-    int tile_bytes;       // bytes of one tile of a row (multiple of 8 KiB, <= kTileBytes)
+    int tile_bytes;       // bytes of one streaming tile (8, 16 or 32 KiB)
     int vec_bytes;        // bytes of a row covered by whole 16-byte vectors
     int vec_elems;        // the same in elements; elements beyond are the row's "tail"
     int tiles_per_unit;   // tiles per row (0 when a row holds no whole vector)
+    int tiles_per_claim;  // tiles one claim covers
+    int claims_per_unit;  // claims per row (>= 1, also for rows without a whole vector)
     int grid;             // CTAs of the streaming kernel
-    int max_slots;        // partial-result slots per unit (>= CTAs that can share one unit)
     int residual_ctas;    // CTAs per rejected row in the residual kernel
-    int64_t num_units;
-    int64_t num_tiles;
+    int64_t num_units;    // rows to stream: B * K * units_per_row
+    int64_t num_claims;   // num_units * claims_per_unit
     int64_t ld_bytes;     // row pitch in bytes
 };
-
-// CTA of the streaming kernel that owns global tile g (CTA c owns [c*NT/G, (c+1)*NT/G)).
-__host__ __device__ __forceinline__ int owner_of_tile(int64_t g, const Geometry& G) {
-    return static_cast<int>(((g + 1) * G.grid - 1) / G.num_tiles);
-}
 
 struct VerifyParams {
     Geometry geo;
@@ -46,15 +45,16 @@ struct VerifyParams {
     const char* draft;    // q logits
     const int32_t* draft_tokens;
     const int32_t* row_len;
-    float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0
+    float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
     int32_t* accept_len;
     int32_t* tokens;
     float* conf;
-    Partial* partials;
-    ResidualTask* tasks;
-    Candidate* candidates;
+    Control* ctl;          // cleared by the host call
+    Partial* partials;     // [num_claims]: unit u owns entries [u * claims_per_unit, ...)
+    ResidualTask* tasks;   // [B]
+    Candidate* candidates; // [B][residual_ctas][2]
     int32_t* status;
 };
 
@@ -198,16 +198,16 @@ __device__ __forceinline__ void absorb_tile(const uint4 (&w)[kVecPerThread], con
     }
 }
 
+// Butterfly over the warp: every lane ends with the combination of all 32 records
+// (same tree in every lane, so the result does not depend on who asks).
 template <bool GREEDY>
-__device__ __forceinline__ void flush_row(const RowState& st, int lane, Partial* out) {
-    float M = st.ref;
+__device__ __forceinline__ Partial warp_combine(float ref, float sum, float best, int index) {
+    float M = ref;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
-    float s = st.sum * ex2_approx(st.ref - M);
+    float s = sum * ex2_approx(ref - M);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-    float best = st.best;
-    int index = st.index;
     if constexpr (GREEDY) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -219,40 +219,42 @@ __device__ __forceinline__ void flush_row(const RowState& st, int lane, Partial*
             }
         }
     }
-    if (lane == 0) {
-        Partial p;
-        p.ref = M;
-        p.sum = s;
-        p.best = best;
-        p.index = index;
-        *out = p;
-    }
+    Partial p;
+    p.ref = M;
+    p.sum = s;
+    p.best = best;
+    p.index = index;
+    return p;
 }
 
-// Position of a unit (a row of one of the two logit tensors) and whether it is in use.
-struct UnitInfo {
-    const char* base;  // first byte of the row
-    bool active;       // position < row_len of its window
+enum : int { kFlagFirst = 1, kFlagLast = 2, kFlagExit = 4 };
+
+// What a ring stage holds; written by the producer before the stage's barrier is armed.
+struct __align__(16) StageDesc {
+    int flags;      // kFlagFirst / kFlagLast tile of its claim; kFlagExit: no more stages
+    int len;        // bytes in the stage (0: the claim has nothing to read)
+    int offset;     // byte offset of the tile in its row
+    unsigned slot;  // claim number (index of its partial)
 };
-__device__ __forceinline__ UnitInfo locate_unit(int64_t u, const VerifyParams& P) {
-    const Geometry& G = P.geo;
-    const int64_t row = (G.units_per_row == 2) ? (u >> 1) : u;
-    const bool is_draft = (G.units_per_row == 2) && (u & 1);
-    const int b = static_cast<int>(row / G.K);
-    const int i = static_cast<int>(row - static_cast<int64_t>(b) * G.K);
-    const int n = P.row_len ? __ldg(P.row_len + b) : G.K;
-    UnitInfo info;
-    info.base = (is_draft ? P.draft : P.target) + row * G.ld_bytes;
-    info.active = i < n;
-    return info;
-}
+
+// Shared memory behind the ring.
+struct SharedControl {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    StageDesc desc[kStages];
+    Partial slots[kSlotSets * kConsumerWarps];  // in-CTA combine buffers
+    unsigned slot_count[kSlotSets];
+    int abort_flag;
+};
+constexpr size_t kSmemBytes = static_cast<size_t>(kStages) * kTileBytes + sizeof(SharedControl);
 
 template <int DT, bool GREEDY>
-__global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_constant__ VerifyParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kTileBytes);
-    uint64_t* empty = full + kStages;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + kStages);
+    SharedControl& sc = *reinterpret_cast<SharedControl*>(smem + kStages * kTileBytes);
+    uint64_t* full = sc.full;
+    uint64_t* empty = sc.empty;
+    volatile int* abort_flag = &sc.abort_flag;
 
     const Geometry& G = P.geo;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -262,40 +264,93 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyP
             mbar_init(full + s, 1);
             mbar_init(empty + s, kConsumerWarps);
         }
-        *abort_flag = 0;
+        for (int s = 0; s < kSlotSets; ++s) sc.slot_count[s] = 0;
+        sc.abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
 
-    const int64_t g_begin = static_cast<int64_t>(blockIdx.x) * G.num_tiles / G.grid;
-    const int64_t g_end = (static_cast<int64_t>(blockIdx.x) + 1) * G.num_tiles / G.grid;
-    int64_t u = g_begin / G.tiles_per_unit;
-    int t = static_cast<int>(g_begin - u * G.tiles_per_unit);
-    int issued = 0;  // tiles put in flight (producer) / taken (consumers); identical sequences
+    int issued = 0;  // stages put in flight (meaningful in the producer thread only)
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // ------------------------------------------------ producer (one thread)
         if (lane == 0) {
-            UnitInfo info = locate_unit(u, P);
-            for (int64_t g = g_begin; g < g_end; ++g) {
-                if (info.active) {
-                    const int s = issued % kStages;
-                    const uint32_t phase = (issued / kStages) & 1;
-                    if (!mbar_wait_bounded(empty + s, phase ^ 1u, abort_flag)) {
-                        *abort_flag = 1;
-                        report(P.status, FEF_ERR_TIMEOUT);
-                        break;
-                    }
-                    const int offset = t * G.tile_bytes;
-                    const int len = min(G.tile_bytes, G.vec_bytes - offset);
-                    mbar_arrive_expect_tx(full + s, static_cast<uint32_t>(len));
-                    bulk_copy_g2s(smem + s * kTileBytes, info.base + offset, static_cast<uint32_t>(len), full + s);
-                    ++issued;
+            bool ok = true;
+            int next_stage = 0;
+            uint32_t next_phase = 0;
+            // the next free stage, or false after a bounded wait ran out
+            auto acquire = [&](int& s) -> bool {
+                s = next_stage;
+                if (!mbar_try_wait(empty + s, next_phase ^ 1u) &&
+                    !mbar_wait_bounded(empty + s, next_phase ^ 1u, abort_flag)) {
+                    *abort_flag = 1;
+                    report(P.status, FEF_ERR_TIMEOUT);
+                    return false;
                 }
-                if (++t == G.tiles_per_unit) {
-                    t = 0;
-                    ++u;
-                    if (g + 1 < g_end) info = locate_unit(u, P);
+                if (++next_stage == kStages) {
+                    next_stage = 0;
+                    next_phase ^= 1u;
+                }
+                return true;
+            };
+
+            // Claims are handed out in row order from a shared counter, so all CTAs stream one
+            // compact, advancing region of memory and finish together.  Tickets are drawn two
+            // ahead so that their round trip never holds up the ring.
+            unsigned long long ticket = atomicAdd(&P.ctl->next_claim, 1ull);
+            unsigned long long ticket_next = atomicAdd(&P.ctl->next_claim, 1ull);
+            while (ok && ticket < static_cast<unsigned long long>(G.num_claims)) {
+                // 32-bit index arithmetic: this thread's instruction count per tile bounds how
+                // fast the ring can be fed
+                const unsigned claim = static_cast<unsigned>(ticket);
+                ticket = ticket_next;
+                ticket_next = atomicAdd(&P.ctl->next_claim, 1ull);
+                const unsigned cpu = static_cast<unsigned>(G.claims_per_unit);
+                const unsigned unit = cpu == 1u ? claim : claim / cpu;
+                const unsigned ci = claim - unit * cpu;
+                const unsigned row = G.units_per_row == 2 ? (unit >> 1) : unit;
+                const bool is_draft = G.units_per_row == 2 && (unit & 1u);
+                const unsigned b = row / static_cast<unsigned>(G.K);
+                const int i = static_cast<int>(row - b * static_cast<unsigned>(G.K));
+                const int n = P.row_len ? __ldg(P.row_len + b) : G.K;
+                const char* base = (is_draft ? P.draft : P.target) + static_cast<int64_t>(row) * G.ld_bytes;
+                const int t_begin = static_cast<int>(ci) * G.tiles_per_claim;
+                const int t_end = min(t_begin + G.tiles_per_claim, G.tiles_per_unit);
+                StageDesc d;
+                d.slot = claim;
+                if (i >= n || t_end <= t_begin) {
+                    // nothing to read: an empty stage still produces the claim's (empty) partial
+                    int s;
+                    if (!(ok = acquire(s))) break;
+                    d.flags = kFlagFirst | kFlagLast;
+                    d.len = 0;
+                    d.offset = 0;
+                    sc.desc[s] = d;
+                    mbar_arrive(full + s);
+                    ++issued;
+                } else {
+                    int offset = t_begin * G.tile_bytes;
+                    for (int t = t_begin; t < t_end; ++t, offset += G.tile_bytes) {
+                        int s;
+                        if (!(ok = acquire(s))) break;
+                        const int len = min(G.tile_bytes, G.vec_bytes - offset);
+                        d.flags = (t == t_begin ? kFlagFirst : 0) | (t == t_end - 1 ? kFlagLast : 0);
+                        d.len = len;
+                        d.offset = offset;
+                        sc.desc[s] = d;
+                        mbar_arrive_expect_tx(full + s, static_cast<uint32_t>(len));
+                        bulk_copy_g2s(smem + s * kTileBytes, base + offset, static_cast<uint32_t>(len), full + s);
+                        ++issued;
+                    }
+                }
+            }
+            if (ok) {
+                int s;
+                if (acquire(s)) {
+                    StageDesc d = {};
+                    d.flags = kFlagExit;
+                    sc.desc[s] = d;
+                    mbar_arrive(full + s);
                 }
             }
         }
@@ -303,55 +358,73 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyP
         // ------------------------------------------------------------ consumers
         RowState st;
         st.reset();
-        bool have_row = false;
-        UnitInfo info = locate_unit(u, P);
-        for (int64_t g = g_begin; g < g_end; ++g) {
-            if (info.active) {
-                have_row = true;
-                const int s = issued % kStages;
-                const uint32_t phase = (issued / kStages) & 1;
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(full + s, phase, abort_flag))) {
-                    *abort_flag = 1;
-                    report(P.status, FEF_ERR_TIMEOUT);
-                    break;
-                }
-                const int offset = t * G.tile_bytes;
-                const int len = min(G.tile_bytes, G.vec_bytes - offset);
-                const unsigned char* stage = smem + s * kTileBytes;
-                uint4 w[kVecPerThread];
-                int at[kVecPerThread];
+        int s = 0;
+        uint32_t phase = 0;
+        int flushes = 0;  // combines done (same sequence in every consumer warp)
+        while (true) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(full + s, phase, abort_flag))) {
+                *abort_flag = 1;
+                report(P.status, FEF_ERR_TIMEOUT);
+                break;
+            }
+            const StageDesc d = sc.desc[s];
+            if (d.flags & kFlagExit) break;
+            const unsigned char* stage = smem + s * kTileBytes;
+
+            if (d.flags & kFlagFirst) st.reset();
+            uint4 w[kVecPerThread];
+            int at[kVecPerThread];
 #pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) {
-                    at[j] = ((j * kConsumerWarps + warp) * 32 + lane) * 16;
-                    if (at[j] < len) w[j] = *reinterpret_cast<const uint4*>(stage + at[j]);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
-                ++issued;
+            for (int j = 0; j < kVecPerThread; ++j) {
+                at[j] = ((j * kConsumerWarps + warp) * 32 + lane) * 16;
+                if (at[j] < d.len) w[j] = *reinterpret_cast<const uint4*>(stage + at[j]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
+            if (++s == kStages) {
+                s = 0;
+                phase ^= 1u;
+            }
+            if (d.len > 0) {
                 if constexpr (GREEDY) {
 #pragma unroll
                     for (int j = 0; j < kVecPerThread; ++j)
-                        if (at[j] < len)
-                            absorb_vector<DT, true>(w[j], (offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
+                        if (at[j] < d.len)
+                            absorb_vector<DT, true>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
                 } else {
-                    if (st.ref == kNoReference && at[0] < len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
-                    if (len == kTileBytes)  // branch-free: the four vectors interleave
-                        absorb_tile<DT, true>(w, at, len, P.c_hi, P.c_lo, st);
+                    if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
+                    if (d.len == kTileBytes)  // branch-free: the four vectors interleave
+                        absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
                     else
-                        absorb_tile<DT, false>(w, at, len, P.c_hi, P.c_lo, st);
+                        absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
                 }
             }
-            if (++t == G.tiles_per_unit || g + 1 == g_end) {
-                if (have_row) {
-                    const int slot = static_cast<int>(blockIdx.x) - owner_of_tile(u * G.tiles_per_unit, G);
-                    flush_row<GREEDY>(st, lane, P.partials + (u * G.max_slots + slot) * kConsumerWarps + warp);
+            if (d.flags & kFlagLast) {
+                // claim finished: warp result -> combine slot; the last warp to arrive folds the 16
+                // records and stores the claim's partial (read by the next kernel)
+                const Partial mine = warp_combine<GREEDY>(st.ref, st.sum, st.best, st.index);
+                const int set = flushes % kSlotSets;
+                ++flushes;
+                unsigned before = 0;
+                if (lane == 0) {
+                    sc.slots[set * kConsumerWarps + warp] = mine;
+                    __threadfence_block();
+                    before = atomicAdd(sc.slot_count + set, 1u);
                 }
-                st.reset();
-                have_row = false;
-                if (t == G.tiles_per_unit) {
-                    t = 0;
-                    ++u;
-                    if (g + 1 < g_end) info = locate_unit(u, P);
+                before = __shfl_sync(0xFFFFFFFFu, before, 0);
+                if (before == kConsumerWarps - 1) {
+                    __threadfence_block();
+                    Partial rec;
+                    rec.ref = kNoReference;
+                    rec.sum = 0.f;
+                    rec.best = -INFINITY;
+                    rec.index = 0x7FFFFFFF;
+                    if (lane < kConsumerWarps) rec = sc.slots[set * kConsumerWarps + lane];
+                    const Partial all = warp_combine<GREEDY>(rec.ref, rec.sum, rec.best, rec.index);
+                    if (lane == 0) {
+                        sc.slot_count[set] = 0;
+                        P.partials[d.slot] = all;
+                    }
                 }
             }
         }
@@ -360,7 +433,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const VerifyP
     __syncthreads();
     // After an abort copies may still be in flight into this CTA's shared memory:
     // give each a bounded chance to land before the CTA retires.
-    if (*abort_flag && warp == kConsumerWarps && lane == 0) {
+    if (*abort_flag && warp == kProducerWarp && lane == 0) {
         const int first = issued > kStages ? issued - kStages : 0;
         for (int k = first; k < issued; ++k) {
             const int s = k % kStages;
@@ -380,39 +453,19 @@ struct RowNorm {
     bool bad;
 };
 
-__device__ __forceinline__ double warp_max(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-    return v;
-}
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
-
-// Combine the streaming kernel's partials of unit u (and the row's tail elements,
-// which the streaming kernel does not touch) into the row's normaliser.  Whole warp.
+// Fold the claims' partials of unit u (and the row's tail elements, which the streaming
+// kernel does not touch) into the row's normaliser.  One thread.
 template <int DT, bool GREEDY>
-__device__ RowNorm finish_row(int64_t u, const char* row, double c, const VerifyParams& P, int lane) {
+__device__ __forceinline__ RowNorm fold_unit(int64_t u, const char* row, double c, const VerifyParams& P) {
     const Geometry& G = P.geo;
-    int nrec = 0;
-    if (G.tiles_per_unit > 0) {
-        const int c_first = owner_of_tile(u * G.tiles_per_unit, G);
-        const int c_last = owner_of_tile((u + 1) * G.tiles_per_unit - 1, G);
-        nrec = (c_last - c_first + 1) * kConsumerWarps;
-    }
-    const Partial* rec = P.partials + u * G.max_slots * kConsumerWarps;
-    const int ntail = G.V - G.vec_elems;
-
-    // each lane folds its records into a running (m, s) pair, then the warp combines
+    const Partial* rec = P.partials + u * G.claims_per_unit;
     double m = -INFINITY, sacc = 0.0;
-    int bad = 0;
+    bool bad = false;
     float best = -INFINITY;
     int index = 0x7FFFFFFF;
-    for (int r = lane; r < nrec; r += 32) {
+    for (int r = 0; r < G.claims_per_unit; ++r) {
         const Partial p = rec[r];
-        if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = 1;
+        if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = true;
         if (p.sum > 0.f) {
             const double pm = p.ref, ps = p.sum;
             if (pm > m) {
@@ -427,10 +480,10 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
             index = p.index;
         }
     }
-    for (int j = lane; j < ntail; j += 32) {
-        const float l = load_logit<DT>(row, G.vec_elems + j);
+    for (int x = G.vec_elems; x < G.V; ++x) {
+        const float l = load_logit<DT>(row, x);
         if (l != l || l == INFINITY) {
-            bad = 1;
+            bad = true;
         } else if (l > -INFINITY) {
             const double pm = static_cast<double>(l) * c;
             if (pm > m) {
@@ -440,137 +493,158 @@ __device__ RowNorm finish_row(int64_t u, const char* row, double c, const Verify
                 sacc += exp2(pm - m);
             }
         }
-        if (GREEDY && better(l, G.vec_elems + j, best, index)) {
+        if (GREEDY && better(l, x, best, index)) {
             best = l;
-            index = G.vec_elems + j;
+            index = x;
         }
     }
-    const double M = warp_max(m);
-    bad = __any_sync(0xFFFFFFFFu, bad);
-    if (GREEDY) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
-            const int oi = __shfl_xor_sync(0xFFFFFFFFu, index, o);
-            if (better(ob, oi, best, index)) {
-                best = ob;
-                index = oi;
-            }
-        }
-    }
-    const double S = warp_sum(m > -INFINITY ? sacc * exp2(m - M) : 0.0);
     RowNorm out;
-    out.M = M;
-    out.S = S;
+    out.M = m;
+    out.S = sacc;
     out.best = best;
     out.index = index;
-    out.bad = bad || !(S > 0.0) || !(S < INFINITY);
+    out.bad = bad || !(sacc > 0.0) || !(sacc < INFINITY);
     return out;
 }
 
-constexpr int kScanMaxWarps = 32;
+constexpr int kScanWarps = 4;  // windows per CTA of the scan kernel
 
+// Acceptance tests, first rejection and outputs (Algorithm 2, "for m = 1..b"): one warp per
+// window, lane l does positions l and l + 32.
 template <int DT, bool GREEDY>
-__global__ void __launch_bounds__(kScanMaxWarps * 32) scan_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_constant__ VerifyParams P) {
     const Geometry& G = P.geo;
-    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
-    const int num_warps = blockDim.x >> 5;
-    const int b = blockIdx.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kRounds = FEF_MAX_K / 32;
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kScanWarps + (threadIdx.x >> 5);
+    if (b >= G.B) return;
     const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
     const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
 
-    __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
-    __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
-    __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
-
-    for (int i = warp; i < n; i += num_warps) {
-        const int64_t row = static_cast<int64_t>(b) * G.K + i;
-        const char* prow = P.target + row * G.ld_bytes;
-        const char* qrow = P.draft + row * G.ld_bytes;
-        const RowNorm np = finish_row<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P, lane);
-        RowNorm nq;
-        nq.bad = false;
-        if constexpr (!GREEDY) nq = finish_row<DT, false>(2 * row + 1, qrow, c, P, lane);
-        if (lane == 0) {
+    // what does not depend on the streaming kernel is fetched before waiting for it
+    int tok[kRounds];
+    double lpx[kRounds], lqx[kRounds];
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        const int i = r * 32 + lane;
+        tok[r] = -1;
+        lpx[r] = lqx[r] = 0.0;
+        if (r * 32 < G.K && i < n) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
             const int x = __ldg(P.draft_tokens + row);
-            int err = 0, accept = 0, alt = -1;
-            float conf = -1.f, conf_alt = -1.f;
-            double kp = 0.0, kq = 0.0;
+            tok[r] = x;
+            if (x >= 0 && x < G.V) {
+                lpx[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
+                if constexpr (!GREEDY) lqx[r] = load_logit<DT>(P.draft + row * G.ld_bytes, x);
+            }
+        }
+    }
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+
+    int alt[kRounds];
+    float cf[kRounds], cf_alt[kRounds];
+    double kp[kRounds], kq[kRounds];
+    unsigned rejected[kRounds];
+    int err = 0;
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        const int i = r * 32 + lane;
+        alt[r] = -1;
+        cf[r] = cf_alt[r] = -1.f;
+        kp[r] = kq[r] = 0.0;
+        bool accept = true;
+        if (r * 32 < G.K && i < n) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
+            const char* prow = P.target + row * G.ld_bytes;
+            const char* qrow = P.draft + row * G.ld_bytes;
+            const int x = tok[r];
+            const RowNorm np = fold_unit<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P);
+            RowNorm nq;
+            nq.bad = false;
+            if constexpr (!GREEDY) nq = fold_unit<DT, false>(2 * row + 1, qrow, c, P);
             if (x < 0 || x >= G.V) {
-                err = FEF_ERR_TOKEN_RANGE;
+                err = max(err, static_cast<int>(FEF_ERR_TOKEN_RANGE));
             } else if (np.bad || nq.bad) {
-                err = FEF_ERR_NONFINITE;
+                err = max(err, static_cast<int>(FEF_ERR_NONFINITE));
             } else {
-                kp = np.M + log2(np.S);
-                const double lpx = load_logit<DT>(prow, x);
-                const double l2pi = lpx * c - kp;  // log2 pi(x)
-                conf = static_cast<float>(exp2(l2pi));
+                kp[r] = np.M + log2(np.S);
+                const double l2pi = lpx[r] * c - kp[r];  // log2 pi(x)
+                cf[r] = static_cast<float>(exp2(l2pi));
                 if constexpr (GREEDY) {
                     accept = (x == np.index);
-                    alt = np.index;
-                    conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
+                    alt[r] = np.index;
+                    cf_alt[r] = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp[r]));
                 } else {
-                    kq = nq.M + log2(nq.S);
-                    const double lqx = load_logit<DT>(qrow, x);
-                    if (lqx == -INFINITY) {
-                        accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
+                    kq[r] = nq.M + log2(nq.S);
+                    if (lqx[r] == -INFINITY) {
+                        accept = lpx[r] > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
                     } else {
-                        const double ratio = exp2(l2pi - (lqx * c - kq));
-                        const uint4 r = philox4x32_10(
+                        const double ratio = exp2(l2pi - (lqx[r] * c - kq[r]));
+                        const uint4 rnd = philox4x32_10(
                             make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), P.step),
                             make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
-                        const double uacc = uniform_from_word(r.x);
+                        const double uacc = uniform_from_word(rnd.x);
                         accept = uacc <= fmin(1.0, ratio);
                     }
                 }
             }
-            s_err[i] = err;
-            s_accept[i] = accept;
-            s_conf[i] = conf;
-            s_conf_alt[i] = conf_alt;
-            s_alt[i] = alt;
-            s_kp[i] = kp;
-            s_kq[i] = kq;
         }
+        rejected[r] = __ballot_sync(0xFFFFFFFFu, !accept);
     }
-    __syncthreads();
+    err = __reduce_max_sync(0xFFFFFFFFu, err);
 
-    int err = 0, a = n;
-    for (int i = 0; i < n; ++i) err = max(err, s_err[i]);
-    for (int i = n - 1; i >= 0; --i)
-        if (!s_accept[i]) a = i;
+    int a = n;
+#pragma unroll
+    for (int r = kRounds - 1; r >= 0; --r)
+        if (rejected[r]) a = r * 32 + __ffs(rejected[r]) - 1;
 
-    for (int i = threadIdx.x; i < G.K; i += blockDim.x) {
-        const int64_t row = static_cast<int64_t>(b) * G.K + i;
-        int tok = -1;
-        float cf = -1.f;
-        if (!err) {
-            if (i < a) {
-                tok = __ldg(P.draft_tokens + row);
-                cf = s_conf[i];
-            } else if (GREEDY && i == a && a < n) {
-                tok = s_alt[i];
-                cf = s_conf_alt[i];
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        const int i = r * 32 + lane;
+        if (i < G.K) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
+            int t = -1;
+            float f = -1.f;
+            if (!err) {
+                if (i < a) {
+                    t = tok[r];
+                    f = cf[r];
+                } else if (GREEDY && i == a && a < n) {
+                    t = alt[r];
+                    f = cf_alt[r];
+                }
             }
+            P.tokens[row] = t;
+            P.conf[row] = f;
         }
-        P.tokens[row] = tok;
-        P.conf[row] = cf;
     }
-    if (threadIdx.x == 0) {
+
+    // the rejected position's normalisers travel with the residual task
+    double kpa = 0.0, kqa = 0.0;
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        const double vp = __shfl_sync(0xFFFFFFFFu, kp[r], a & 31);
+        const double vq = __shfl_sync(0xFFFFFFFFu, kq[r], a & 31);
+        if ((a >> 5) == r) {
+            kpa = vp;
+            kqa = vq;
+        }
+    }
+    if (lane == 0) {
         P.accept_len[b] = err ? -1 : a;
         if (err) report(P.status, err);
         ResidualTask task;
         task.pos = (!GREEDY && !err && a < n) ? a : -1;
         task.arrivals = 0u;
-        task.kp = task.pos >= 0 ? s_kp[a] : 0.0;
-        task.kq = task.pos >= 0 ? s_kq[a] : 0.0;
+        task.kp = task.pos >= 0 ? kpa : 0.0;
+        task.kq = task.pos >= 0 ? kqa : 0.0;
         P.tasks[b] = task;
     }
 }
 
 // ============================================================= residual ====
 constexpr int kResidualThreads = 256;
+constexpr int kResidualBatch = 4;   // vector pairs a thread has in flight
 constexpr int kMaxResidualCtas = kResidualThreads / 2;  // the last CTA looks at 2 candidates per CTA
 
 // -ln(u) for u = ((word >> 9) + 0.5) * 2^-23, accurate also when u is close to 1.
@@ -649,7 +723,7 @@ __device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __grid_constant__ VerifyParams P) {
     constexpr int N = Elem<DT>::kPerVec;
     const Geometry& G = P.geo;
     cudaGridDependencySynchronize();  // the scan kernel's tasks must be complete and visible
@@ -667,29 +741,43 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const Ver
     Top2 top;
     top.clear();
 
-    // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x)
+    // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x).  A thread's loads
+    //      are all issued before the arithmetic, and every group of four ids gets its Philox call
+    //      whether or not it holds a positive r (no branches between independent chains).
     const int nvec = G.vec_elems / N;
     const int v_begin = static_cast<int>(static_cast<int64_t>(part) * nvec / parts);
     const int v_end = static_cast<int>(static_cast<int64_t>(part + 1) * nvec / parts);
-    for (int vec = v_begin + threadIdx.x; vec < v_end; vec += kResidualThreads) {
-        float lp[N], lq[N], r[N];
-        unpack<DT>(ld_global_nc_v4(prow + static_cast<int64_t>(vec) * 16), lp);
-        unpack<DT>(ld_global_nc_v4(qrow + static_cast<int64_t>(vec) * 16), lq);
+    for (int v0 = v_begin; v0 < v_end; v0 += kResidualThreads * kResidualBatch) {
+        uint4 wp[kResidualBatch], wq[kResidualBatch];
+        int vec[kResidualBatch];
 #pragma unroll
-        for (int i = 0; i < N; ++i)
-            r[i] = exp2_scaled<DT>(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq[i], P.c_hi, P.c_lo, kq);
+        for (int j = 0; j < kResidualBatch; ++j) {
+            vec[j] = v0 + j * kResidualThreads + static_cast<int>(threadIdx.x);
+            if (vec[j] < v_end) {
+                wp[j] = ld_global_nc_v4(prow + static_cast<int64_t>(vec[j]) * 16);
+                wq[j] = ld_global_nc_v4(qrow + static_cast<int64_t>(vec[j]) * 16);
+            }
+        }
 #pragma unroll
-        for (int g4 = 0; g4 < N / 4; ++g4) {
-            const float rmax = fmaxf(fmaxf(r[4 * g4], r[4 * g4 + 1]), fmaxf(r[4 * g4 + 2], r[4 * g4 + 3]));
-            if (rmax > 0.f) {
-                const int x0 = vec * N + 4 * g4;
+        for (int j = 0; j < kResidualBatch; ++j) {
+            if (vec[j] >= v_end) continue;
+            float lp[N], lq[N], r[N];
+            unpack<DT>(wp[j], lp);
+            unpack<DT>(wq[j], lq);
+#pragma unroll
+            for (int i = 0; i < N; ++i)
+                r[i] = exp2_scaled<DT>(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq[i], P.c_hi, P.c_lo, kq);
+#pragma unroll
+            for (int g4 = 0; g4 < N / 4; ++g4) {
+                const int x0 = vec[j] * N + 4 * g4;
                 const uint4 w = philox4x32_10(
                     make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
                 const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const float ri = r[4 * g4 + i];
-                    if (ri > 0.f) top.offer(__fdividef(ri, neg_log_uniform(words[i])), x0 + i);
+                    const float wi = ri > 0.f ? __fdividef(ri, neg_log_uniform(words[i])) : 0.f;
+                    if (wi >= top.w2 && wi > 0.f) top.offer(wi, x0 + i);
                 }
             }
         }
@@ -801,6 +889,9 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const Ver
 static int g_sm_count[64];
 static bool g_attr_done[64][4];
 
+constexpr int kClaimsPerCta = 6;             // streaming claims a CTA should get at least, size permitting
+constexpr int kMaxClaimBytes = 1 << 20;      // and at most this many bytes per claim (a whole row of the usual sizes)
+
 static int sm_count_of_current_device(int* device_out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
@@ -827,22 +918,38 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool gr
     G.vec_bytes = static_cast<int>((static_cast<int64_t>(V) * esize) / 16 * 16);
     G.vec_elems = G.vec_bytes / esize;
     G.num_units = static_cast<int64_t>(B) * K * G.units_per_row;
-    const int64_t cta_target = sm_count;
-    // the largest tile that still leaves every CTA several tiles to pipeline
+
+    // streaming claims: large enough to amortise their bookkeeping, small enough that every
+    // CTA gets several and the last ones end close together
+    int64_t claim_target = G.num_units * G.vec_bytes / (static_cast<int64_t>(sm_count) * kClaimsPerCta);
+    if (claim_target > kMaxClaimBytes) claim_target = kMaxClaimBytes;
+    if (claim_target < 8192) claim_target = 8192;
     G.tile_bytes = kTileBytes;
-    while (G.tile_bytes > 8192 &&
-           G.num_units * ((G.vec_bytes + G.tile_bytes - 1) / G.tile_bytes) < 8 * cta_target)
-        G.tile_bytes >>= 1;
+    while (G.tile_bytes > 8192 && G.tile_bytes > claim_target) G.tile_bytes >>= 1;
     G.tiles_per_unit = (G.vec_bytes + G.tile_bytes - 1) / G.tile_bytes;
-    G.num_tiles = G.num_units * G.tiles_per_unit;
-    G.grid = static_cast<int>(G.num_tiles < cta_target ? G.num_tiles : cta_target);
-    if (G.grid < 1) G.grid = 1;
-    const int64_t min_tiles_per_cta = G.num_tiles > 0 ? G.num_tiles / G.grid : 1;
-    G.max_slots = G.tiles_per_unit > 0 ? static_cast<int>((G.tiles_per_unit - 1) / min_tiles_per_cta) + 2 : 1;
-    int parts = (6 * sm_count + B - 1) / B;
+    if (G.tiles_per_unit > 0) {
+        int tpc = static_cast<int>(claim_target / G.tile_bytes);
+        if (tpc < 1) tpc = 1;
+        if (tpc > G.tiles_per_unit) tpc = G.tiles_per_unit;
+        G.claims_per_unit = (G.tiles_per_unit + tpc - 1) / tpc;
+        G.tiles_per_claim = (G.tiles_per_unit + G.claims_per_unit - 1) / G.claims_per_unit;  // even split
+        G.claims_per_unit = (G.tiles_per_unit + G.tiles_per_claim - 1) / G.tiles_per_claim;
+    } else {
+        G.tiles_per_claim = 1;
+        G.claims_per_unit = 1;
+    }
+    G.num_claims = G.num_units * G.claims_per_unit;
+    if (G.num_claims >= (1ll << 31)) return false;  // claim numbers are handled as 32-bit values
+    G.grid = static_cast<int>(G.num_claims < sm_count ? G.num_claims : sm_count);
+
+    // residual kernel: CTAs per rejected row, each thread up to kResidualBatch vector pairs
+    // (fewer when few windows would leave SMs idle)
     const int nvec = G.vec_bytes / 16;
-    const int max_parts_by_size = nvec / kResidualThreads > 0 ? nvec / kResidualThreads : 1;
-    if (parts > max_parts_by_size) parts = max_parts_by_size;
+    int per_thread = kResidualBatch;
+    while (per_thread > 1 &&
+           static_cast<int64_t>(B) * ((nvec + kResidualThreads * per_thread - 1) / (kResidualThreads * per_thread)) < 2 * sm_count)
+        per_thread >>= 1;
+    int parts = (nvec + kResidualThreads * per_thread - 1) / (kResidualThreads * per_thread);
     if (parts > kMaxResidualCtas) parts = kMaxResidualCtas;
     if (parts < 1) parts = 1;
     G.residual_ctas = parts;
@@ -850,29 +957,21 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool gr
     return true;
 }
 
+// Scratch layout: control (cleared on every call), partials, tasks, candidates (every value
+// written before it is read).
 struct WorkspaceLayout {
-    size_t partials, tasks, candidates, total;
+    size_t control, zero_bytes, partials, tasks, candidates, total;
 };
 static size_t round256(size_t n) { return (n + 255) & ~static_cast<size_t>(255); }
 static WorkspaceLayout layout_of(const Geometry& G) {
     WorkspaceLayout L;
-    L.partials = 0;
-    L.tasks = round256(static_cast<size_t>(G.num_units) * G.max_slots * kConsumerWarps * sizeof(Partial));
+    L.control = 0;
+    L.zero_bytes = round256(sizeof(Control));
+    L.partials = L.zero_bytes;
+    L.tasks = L.partials + round256(static_cast<size_t>(G.num_claims) * sizeof(Partial));
     L.candidates = L.tasks + round256(static_cast<size_t>(G.B) * sizeof(ResidualTask));
     L.total = L.candidates + round256(static_cast<size_t>(G.B) * kMaxResidualCtas * 2 * sizeof(Candidate));
     return L;
-}
-
-template <typename Kernel>
-static cudaError_t allow_large_smem(Kernel k, int dev, int which, size_t bytes) {
-    if (g_attr_done[dev][which]) return cudaSuccess;
-    const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
-    if (e == cudaSuccess) g_attr_done[dev][which] = true;
-    return e;
-}
-
-static void mark(void* const* events, int which, cudaStream_t stream) {
-    if (events && events[which]) cudaEventRecord(static_cast<cudaEvent_t>(events[which]), stream);
 }
 
 // Launch with programmatic dependent launch: the grid may be scheduled while its
@@ -895,33 +994,23 @@ static cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 blo
 }
 
 template <int DT, bool GREEDY>
-static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream, void* const* events) {
+static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream) {
     const Geometry& G = P.geo;
-    const size_t smem = static_cast<size_t>(kStages) * kTileBytes + 2 * kStages * sizeof(uint64_t) + 16;
-    const bool timed = events != nullptr;  // event records between kernels rule out dependent launches
-    mark(events, 0, stream);
-    if (G.num_tiles > 0) {
-        cudaError_t e = allow_large_smem(stream_kernel<DT, GREEDY>, dev, DT * 2 + (GREEDY ? 1 : 0), smem);
+    const int which = DT * 2 + (GREEDY ? 1 : 0);
+    if (!g_attr_done[dev][which]) {
+        const cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(kSmemBytes));
         if (e != cudaSuccess) return e;
-        stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, smem, stream>>>(P);
+        g_attr_done[dev][which] = true;
     }
-    mark(events, 1, stream);
-    const int scan_threads = 32 * (G.K < kScanMaxWarps ? G.K : kScanMaxWarps);
-    cudaError_t e;
-    if (timed)
-        scan_kernel<DT, GREEDY><<<G.B, scan_threads, 0, stream>>>(P), e = cudaGetLastError();
-    else
-        e = launch_dependent(scan_kernel<DT, GREEDY>, dim3(G.B), dim3(scan_threads), 0, stream, P);
+    stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, kSmemBytes, stream>>>(P);
+    cudaError_t e = launch_dependent(scan_kernel<DT, GREEDY>, dim3((G.B + kScanWarps - 1) / kScanWarps),
+                                     dim3(kScanWarps * 32), 0, stream, P);
     if (e != cudaSuccess) return e;
-    mark(events, 2, stream);
     if (!GREEDY) {
-        if (timed)
-            residual_kernel<DT><<<dim3(G.residual_ctas, G.B), kResidualThreads, 0, stream>>>(P), e = cudaGetLastError();
-        else
-            e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
+        e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
         if (e != cudaSuccess) return e;
     }
-    mark(events, 3, stream);
     return cudaGetLastError();
 }
 
@@ -954,12 +1043,11 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
     return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
 }
 
-fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
-                                    const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
-                                    int64_t ld, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
-                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
-                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
-                                    void* const* stage_events) {
+fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* cuda_stream) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -1008,6 +1096,7 @@ fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target
     P.tokens = tokens;
     P.conf = conf;
     char* ws = static_cast<char*>(workspace);
+    P.ctl = reinterpret_cast<Control*>(ws + L.control);
     P.partials = reinterpret_cast<Partial*>(ws + L.partials);
     P.tasks = reinterpret_cast<ResidualTask*>(ws + L.tasks);
     P.candidates = reinterpret_cast<Candidate*>(ws + L.candidates);
@@ -1016,24 +1105,14 @@ fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (device_status && cudaMemsetAsync(device_status, 0, sizeof(int32_t), stream) != cudaSuccess)
         return FEF_ERR_CUDA;
+    // the claim counter of the call starts at zero; nothing else in the scratch needs a defined value
+    if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return FEF_ERR_CUDA;
     cudaError_t e;
     if (dt == FEF_F32)
-        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream, stage_events)
-                   : launch_all<FEF_F32, false>(P, dev, stream, stage_events);
+        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream) : launch_all<FEF_F32, false>(P, dev, stream);
     else
-        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream, stage_events)
-                   : launch_all<FEF_BF16, false>(P, dev, stream, stage_events);
+        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream) : launch_all<FEF_BF16, false>(P, dev, stream);
     return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
-}
-
-fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
-                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
-                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
-                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
-                           int32_t* device_status, void* cuda_stream) {
-    return fef_spec_verify_profiled(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt,
-                                    temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes,
-                                    device_status, cuda_stream, nullptr);
 }
 
 // ---- host-buffer variant: layout of the caller's device arena
@@ -1143,9 +1222,10 @@ fef_status fef_spec_verify_static(const void* draft_logits, const void* target_l
         if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return FEF_ERR_CUDA;
         g_static_scratch_address[dev] = scratch;
     }
-    // Nothing in the scratch has to start at zero: the streaming kernel overwrites every partial
-    // the scan reads, and the scan rewrites every window's task (arrival counter included)
-    // before the residual kernel looks at it, so leftovers of earlier calls are never read.
+    // The array keeps what the previous call left.  fef_spec_verify clears the part that must
+    // start at zero (the streaming kernel's claim counter) on the stream before its kernels;
+    // every other value is written before it is read (the scan kernel rewrites every window's
+    // task, arrival counter included), so leftovers of earlier calls are never used.
     return fef_spec_verify(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt, temperature, seed,
                            step, accept_len, tokens, conf, scratch, FEF_STATIC_SCRATCH_BYTES, device_status,
                            cuda_stream);

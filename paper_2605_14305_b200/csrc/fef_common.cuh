@@ -70,9 +70,10 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key) {
     constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, ctr.x), lo0 = M0 * ctr.x;
-        const uint32_t hi1 = __umulhi(M1, ctr.z), lo1 = M1 * ctr.z;
-        ctr = make_uint4(hi1 ^ ctr.y ^ key.x, lo1, hi0 ^ ctr.w ^ key.y, lo0);
+        const uint64_t p0 = static_cast<uint64_t>(M0) * ctr.x;  // one wide multiply gives both halves
+        const uint64_t p1 = static_cast<uint64_t>(M1) * ctr.z;
+        ctr = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ ctr.y ^ key.x, static_cast<uint32_t>(p1),
+                         static_cast<uint32_t>(p0 >> 32) ^ ctr.w ^ key.y, static_cast<uint32_t>(p0));
         key.x += W0;
         key.y += W1;
     }

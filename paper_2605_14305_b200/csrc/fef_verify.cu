@@ -647,13 +647,16 @@ constexpr int kResidualThreads = 256;
 constexpr int kResidualBatch = 4;   // vector pairs a thread has in flight
 constexpr int kMaxResidualCtas = kResidualThreads / 2;  // the last CTA looks at 2 candidates per CTA
 
-// -ln(u) for u = ((word >> 9) + 0.5) * 2^-23, accurate also when u is close to 1.
-__device__ __forceinline__ float neg_log_uniform(uint32_t word) {
-    const float k = static_cast<float>(word >> 9);
-    const float u = (k + 0.5f) * (1.0f / 8388608.0f);
-    const float t = (8388607.5f - k) * (1.0f / 8388608.0f);  // 1 - u, exact
+// For u = ((word >> 9) + 0.5) * 2^-23:  t = 1 - u (exact in binary32) and -ln(u), accurate
+// also when u is close to 1.  Always -ln(u) > t.
+__device__ __forceinline__ float one_minus_uniform(uint32_t word) {
+    // k = word >> 9;  2^23 + (2^23 - 1 - k) assembled in the mantissa, then one exact multiply-add
+    const float f = __uint_as_float(0x4B000000u | (~word >> 9));
+    return fmaf(f, 1.0f / 8388608.0f, -(1.0f - 1.0f / 16777216.0f));
+}
+__device__ __forceinline__ float neg_log_uniform(float t) {
     const float series = t * fmaf(t, fmaf(t, fmaf(t, 0.25f, 1.0f / 3.0f), 0.5f), 1.0f);
-    const float direct = -0.6931471805599453f * lg2_approx(u);
+    const float direct = -0.6931471805599453f * lg2_approx(1.0f - t);  // 1 - t = u exactly
     return t < 0.015625f ? series : direct;
 }
 
@@ -673,6 +676,16 @@ struct Top2 {
         } else if (better(w, x, w2, x2)) {
             w2 = w;
             x2 = x;
+        }
+    }
+    // best two of the whole warp, in every lane
+    __device__ __forceinline__ void warp_merge() {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ow1 = __shfl_xor_sync(0xFFFFFFFFu, w1, o), ow2 = __shfl_xor_sync(0xFFFFFFFFu, w2, o);
+            const int ox1 = __shfl_xor_sync(0xFFFFFFFFu, x1, o), ox2 = __shfl_xor_sync(0xFFFFFFFFu, x2, o);
+            offer(ow1, ox1);
+            offer(ow2, ox2);
         }
     }
 };
@@ -740,10 +753,15 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
 
     Top2 top;
     top.clear();
+    // A lower bound of the CTA's second-best weight so far (bits of a non-negative float).  An id
+    // whose weight cannot exceed it is dropped after one multiply; a stale value is only less sharp.
+    __shared__ unsigned s_floor;
+    if (threadIdx.x == 0) s_floor = 0u;
+    __syncthreads();
+    bool inserted = false;
 
     // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x).  A thread's loads
-    //      are all issued before the arithmetic, and every group of four ids gets its Philox call
-    //      whether or not it holds a positive r (no branches between independent chains).
+    //      are all issued before the arithmetic; every group of four ids gets its Philox call.
     const int nvec = G.vec_elems / N;
     const int v_begin = static_cast<int>(static_cast<int64_t>(part) * nvec / parts);
     const int v_end = static_cast<int>(static_cast<int64_t>(part + 1) * nvec / parts);
@@ -753,14 +771,17 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
 #pragma unroll
         for (int j = 0; j < kResidualBatch; ++j) {
             vec[j] = v0 + j * kResidualThreads + static_cast<int>(threadIdx.x);
+            // a lane beyond the end works on -inf logits (r = 0 never qualifies), so the warp stays whole
+            constexpr uint32_t kMinusInf = DT == FEF_F32 ? 0xFF800000u : 0xFF80FF80u;
+            wp[j] = wq[j] = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
             if (vec[j] < v_end) {
                 wp[j] = ld_global_nc_v4(prow + static_cast<int64_t>(vec[j]) * 16);
                 wq[j] = ld_global_nc_v4(qrow + static_cast<int64_t>(vec[j]) * 16);
             }
         }
+        float floor_w = fmaxf(top.w2, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&s_floor)));
 #pragma unroll
         for (int j = 0; j < kResidualBatch; ++j) {
-            if (vec[j] >= v_end) continue;
             float lp[N], lq[N], r[N];
             unpack<DT>(wp[j], lp);
             unpack<DT>(wq[j], lq);
@@ -772,14 +793,28 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
                 const int x0 = vec[j] * N + 4 * g4;
                 const uint4 w = philox4x32_10(
                     make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
-                const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float ri = r[4 * g4 + i];
-                    const float wi = ri > 0.f ? __fdividef(ri, neg_log_uniform(words[i])) : 0.f;
-                    if (wi >= top.w2 && wi > 0.f) top.offer(wi, x0 + i);
+                // w = r / (-ln u) < r / t: nearly every id is ruled out by one multiply and compare;
+                // the vote keeps the rare rest out of the straight-line code
+                const float t0 = one_minus_uniform(w.x), t1 = one_minus_uniform(w.y);
+                const float t2 = one_minus_uniform(w.z), t3 = one_minus_uniform(w.w);
+                const bool q0 = r[4 * g4] > floor_w * t0, q1 = r[4 * g4 + 1] > floor_w * t1;
+                const bool q2 = r[4 * g4 + 2] > floor_w * t2, q3 = r[4 * g4 + 3] > floor_w * t3;
+                if (__any_sync(0xFFFFFFFFu, q0 || q1 || q2 || q3)) {
+                    if (q0) top.offer(__fdividef(r[4 * g4], neg_log_uniform(t0)), x0);
+                    if (q1) top.offer(__fdividef(r[4 * g4 + 1], neg_log_uniform(t1)), x0 + 1);
+                    if (q2) top.offer(__fdividef(r[4 * g4 + 2], neg_log_uniform(t2)), x0 + 2);
+                    if (q3) top.offer(__fdividef(r[4 * g4 + 3], neg_log_uniform(t3)), x0 + 3);
+                    floor_w = fmaxf(floor_w, top.w2);
+                    inserted = inserted || q0 || q1 || q2 || q3;
                 }
             }
+        }
+        if (__any_sync(0xFFFFFFFFu, inserted)) {
+            // some lane took an id: the warp's second-best weight may have risen; tell the CTA
+            Top2 merged = top;
+            merged.warp_merge();
+            if ((threadIdx.x & 31) == 0 && merged.w2 > 0.f) atomicMax(&s_floor, __float_as_uint(merged.w2));
+            inserted = false;
         }
     }
     // tail elements (beyond the last whole vector) belong to part 0
@@ -791,19 +826,13 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
                 const uint4 w = philox4x32_10(
                     make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), ub, upos, P.step), key);
                 const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
-                top.offer(__fdividef(r, neg_log_uniform(word)), x);
+                top.offer(__fdividef(r, neg_log_uniform(one_minus_uniform(word))), x);
             }
         }
     }
 
     // ---- CTA-wide best two
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ow1 = __shfl_xor_sync(0xFFFFFFFFu, top.w1, o), ow2 = __shfl_xor_sync(0xFFFFFFFFu, top.w2, o);
-        const int ox1 = __shfl_xor_sync(0xFFFFFFFFu, top.x1, o), ox2 = __shfl_xor_sync(0xFFFFFFFFu, top.x2, o);
-        top.offer(ow1, ox1);
-        top.offer(ow2, ox2);
-    }
+    top.warp_merge();
     __shared__ Top2 s_top[kResidualThreads / 32];
     __shared__ int s_last;
     __shared__ double s_score[kResidualThreads / 32];

@@ -758,7 +758,6 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
     __shared__ unsigned s_floor;
     if (threadIdx.x == 0) s_floor = 0u;
     __syncthreads();
-    bool inserted = false;
 
     // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x).  A thread's loads
     //      are all issued before the arithmetic; every group of four ids gets its Philox call.
@@ -793,8 +792,8 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
                 const int x0 = vec[j] * N + 4 * g4;
                 const uint4 w = philox4x32_10(
                     make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
-                // w = r / (-ln u) < r / t: nearly every id is ruled out by one multiply and compare;
-                // the vote keeps the rare rest out of the straight-line code
+                // w = r / (-ln u) < r / t: once the floor is up, nearly every id is ruled out by one
+                // multiply and compare; the vote keeps the rare rest out of the straight-line code
                 const float t0 = one_minus_uniform(w.x), t1 = one_minus_uniform(w.y);
                 const float t2 = one_minus_uniform(w.z), t3 = one_minus_uniform(w.w);
                 const bool q0 = r[4 * g4] > floor_w * t0, q1 = r[4 * g4 + 1] > floor_w * t1;
@@ -804,18 +803,18 @@ __global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __g
                     if (q1) top.offer(__fdividef(r[4 * g4 + 1], neg_log_uniform(t1)), x0 + 1);
                     if (q2) top.offer(__fdividef(r[4 * g4 + 2], neg_log_uniform(t2)), x0 + 2);
                     if (q3) top.offer(__fdividef(r[4 * g4 + 3], neg_log_uniform(t3)), x0 + 3);
-                    floor_w = fmaxf(floor_w, top.w2);
-                    inserted = inserted || q0 || q1 || q2 || q3;
                 }
             }
+            // raise the floor: any lane's second-best weight bounds the CTA's second best from below
+            floor_w = fmaxf(floor_w, __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(top.w2))));
+            if (j == 0 && v0 == v_begin) {
+                // after the first vector of every thread the whole CTA shares what it has found
+                if ((threadIdx.x & 31) == 0) atomicMax(&s_floor, __float_as_uint(floor_w));
+                __syncthreads();
+                floor_w = fmaxf(floor_w, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&s_floor)));
+            }
         }
-        if (__any_sync(0xFFFFFFFFu, inserted)) {
-            // some lane took an id: the warp's second-best weight may have risen; tell the CTA
-            Top2 merged = top;
-            merged.warp_merge();
-            if ((threadIdx.x & 31) == 0 && merged.w2 > 0.f) atomicMax(&s_floor, __float_as_uint(merged.w2));
-            inserted = false;
-        }
+        if ((threadIdx.x & 31) == 0) atomicMax(&s_floor, __float_as_uint(floor_w));
     }
     // tail elements (beyond the last whole vector) belong to part 0
     if (part == 0) {

@@ -37,7 +37,7 @@ METRIC = "verified draft positions/sec"
 UNIT = "positions/s"
 REMASK_L = 1024
 FALLBACK_HBM_GBS = 6650.0
-TRAFFIC_FILE = os.path.join(ROOT, "profiles", "verify_kernel_bf16_ncu.md")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "verify_kernels_B16_bf16_ncu.md")
 
 
 # ------------------------------------------------------------------ helpers ----
@@ -309,7 +309,7 @@ def run_native(args):
     peak, peak_src = _measured_peak()
     row_bytes = (2 if w.temperature > 0 else 1) * w.V * w.logit_bytes
     stream_bytes = w.B * w.K * row_bytes
-    roof = {"bound": "hbm", "kernel": "verify_kernel", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
+    roof = {"bound": "hbm", "kernel": "fef_spec_verify (stream_kernel + scan_kernel + residual_kernel)", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
             "traffic": _ncu_traffic(), "algorithmic_bytes_per_launch": stream_bytes}
     if not args.no_call_events and call_ms[0] > 0:
         roof["achieved"] = stream_bytes / (call_ms[0] * 1e-3) / 1e9
@@ -318,8 +318,8 @@ def run_native(args):
         roof["ms_per_launch"] = call_ms[0]
         roof["call_ms"] = {"fef_spec_verify": call_ms[0], "fef_remask_select": call_ms[1]}
         roof["timed"] = ("second pass over the same K steps with CUDA events around each call; the verification "
-                         "call is one kernel (plus the clearing of its counters), and every row is counted once "
-                         "although the rejected rows are read a second time")
+                         "call is three kernels (plus the clearing of its claim counter), and every row is counted "
+                         "once although the rejected rows are read a second time")
     else:
         roof["achieved"], roof["frac"] = None, None
     call_bytes = synth.algorithmic_bytes(w, rejected_rows=rejected)
@@ -334,7 +334,7 @@ def run_native(args):
         "e2e": {"value": positions_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "api": "fef_spec_verify_host + fef_remask_select_host (pinned host buffers)"},
-        "gpu_launches": steps * 2,
+        "gpu_launches": steps * 4,
         "clocks": sampler.result(),
         "cpu_baseline": cpu_baseline,
         "parity_vs_oracle": parity,

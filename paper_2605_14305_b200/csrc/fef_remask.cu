@@ -3,8 +3,11 @@
 //
 // One CTA per batch row.  Every position becomes a 64-bit key
 // (order-preserving image of the confidence << 32 | index), non-candidates get
-// the largest key, and the keys are sorted in shared memory with a bitonic
-// network; the first min(k, candidates) keys are the answer.
+// the largest key.  For k <= 32 (the usual re-mask counts) each warp keeps the
+// 32 smallest keys of its share of the row in its lanes (bitonic sort and merge
+// by shuffles, no shared memory in the loop) and one warp merges the warps'
+// lists; for larger k the keys are sorted in shared memory with a bitonic
+// network.  The first min(k, candidates) keys are the answer.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -71,6 +74,79 @@ __global__ void __launch_bounds__(kRemaskThreads) remask_kernel(const float* __r
     if (threadIdx.x == 0) count[b] = n;
 }
 
+// ---- k <= 32: warp-level selection
+constexpr int kSmallThreads = 256;
+constexpr int kSmallWarps = kSmallThreads / 32;
+
+// Ascending bitonic sort of the warp's 32 keys (one per lane).
+__device__ __forceinline__ uint64_t warp_sort32(uint64_t v, int lane) {
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const uint64_t other = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
+            const bool ascending = (lane & size) == 0;
+            const bool lower = (lane & stride) == 0;
+            const uint64_t lo = v < other ? v : other, hi = v < other ? other : v;
+            v = (lower == ascending) ? lo : hi;
+        }
+    }
+    return v;
+}
+// The 32 smallest of two ascending lists (a, b: one key per lane each), ascending again.
+__device__ __forceinline__ uint64_t warp_merge_low32(uint64_t a, uint64_t b, int lane) {
+    const uint64_t reversed = __shfl_sync(0xFFFFFFFFu, b, 31 - lane);
+    uint64_t v = a < reversed ? a : reversed;  // bitonic, holds the 32 smallest of the union
+#pragma unroll
+    for (int stride = 16; stride > 0; stride >>= 1) {
+        const uint64_t other = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
+        const uint64_t lo = v < other ? v : other, hi = v < other ? other : v;
+        v = (lane & stride) == 0 ? lo : hi;
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(kSmallThreads) remask_small_kernel(const float* __restrict__ conf,
+                                                                     const uint8_t* __restrict__ mask, int L, int k,
+                                                                     int32_t* __restrict__ positions,
+                                                                     int32_t* __restrict__ count) {
+    __shared__ uint64_t s_keys[kSmallWarps][32];
+    __shared__ int s_total;
+    cudaGridDependencySynchronize();  // conf may come straight from a verification call on this stream
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float* c = conf + static_cast<int64_t>(b) * L;
+    const uint8_t* m = mask + static_cast<int64_t>(b) * L;
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+
+    uint64_t best = ~0ull;  // the warp's 32 smallest keys so far, ascending over the lanes
+    int mine = 0;
+    for (int base = warp * 32; base < L; base += kSmallThreads) {
+        const int i = base + lane;
+        uint64_t key = ~0ull;
+        if (i < L && m[i] != 0) {
+            key = (static_cast<uint64_t>(order_key(c[i])) << 32) | static_cast<uint32_t>(i);
+            ++mine;
+        }
+        best = warp_merge_low32(best, warp_sort32(key, lane), lane);
+    }
+    mine += __shfl_xor_sync(0xFFFFFFFFu, mine, 16);
+    mine += __shfl_xor_sync(0xFFFFFFFFu, mine, 8);
+    mine += __shfl_xor_sync(0xFFFFFFFFu, mine, 4);
+    mine += __shfl_xor_sync(0xFFFFFFFFu, mine, 2);
+    mine += __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
+    if (lane == 0 && mine) atomicAdd(&s_total, mine);
+    s_keys[warp][lane] = best;
+    __syncthreads();
+    if (warp != 0) return;
+    for (int w = 1; w < kSmallWarps; ++w) best = warp_merge_low32(best, s_keys[w][lane], lane);
+    const int total = s_total;
+    const int n = total < k ? total : k;
+    if (lane < k) positions[static_cast<int64_t>(b) * k + lane] = lane < n ? static_cast<int32_t>(best & 0xFFFFFFFFu) : -1;
+    if (lane == 0) count[b] = n;
+}
+
 static bool g_remask_attr_done[64];
 
 }  // namespace fef
@@ -82,6 +158,22 @@ extern "C" fef_status fef_remask_select(const float* conf, const uint8_t* mask, 
     if (k > 0 && !positions) return FEF_ERR_INVALID_ARG;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FEF_ERR_CUDA;
+    // programmatic dependent launch: the grid may be scheduled while the previous kernel on the
+    // stream drains; the kernel waits for it before reading anything
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (k <= 32) {
+        cfg.blockDim = dim3(kSmallThreads);
+        cfg.dynamicSmemBytes = 0;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, remask_small_kernel, conf, mask, L, k, positions, count);
+        return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    }
     int n_sort = 2;
     while (n_sort < L) n_sort <<= 1;
     const size_t smem = static_cast<size_t>(n_sort) * sizeof(uint64_t);
@@ -91,18 +183,8 @@ extern "C" fef_status fef_remask_select(const float* conf, const uint8_t* mask, 
             return FEF_ERR_CUDA;
         g_remask_attr_done[dev] = true;
     }
-    // programmatic dependent launch: the grid may be scheduled while the previous kernel on the
-    // stream drains; the kernel waits for it before reading anything
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(B);
     cfg.blockDim = dim3(kRemaskThreads);
     cfg.dynamicSmemBytes = smem;
-    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, remask_kernel, conf, mask, L, k, n_sort, positions, count);
     return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }

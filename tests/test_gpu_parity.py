@@ -273,7 +273,8 @@ def test_far_apart_laws_reject_at_once_and_wide_dynamic_range(fef):
 
 
 @pytest.mark.parametrize("B,L,k", [(1, 1, 1), (3, 17, 5), (8, 256, 8), (2, 1024, 2), (4, 33, 40), (2, 9, 0),
-                                   (2, 8192, 8), (64, 1024, 8), (1, 5000, 5000)])
+                                   (2, 8192, 8), (64, 1024, 8), (1, 5000, 5000), (3, 100, 32), (3, 100, 33), (2, 20, 32),
+                                   (5, 2049, 31)])
 def test_remask_select_matches_oracle(fef, B, L, k):
     g = torch.Generator(device="cuda").manual_seed(B * 1000 + L)
     conf = torch.rand((B, L), generator=g, device="cuda")

@@ -200,6 +200,56 @@ __device__ __forceinline__ void absorb_tile(const uint4 (&w)[kVecPerThread], con
 
 // Butterfly over the warp: every lane ends with the combination of all 32 records
 // (same tree in every lane, so the result does not depend on who asks).
+// Greedy mode: largest logit of the thread's share and its lowest index.  The exact update
+// (unpack, compare, find the index) runs only for a vector that holds an element >= the warp's
+// running maximum (refreshed once per tile); anything smaller cannot be the row's arg-max, and
+// equal elements still go through the exact update, so the lowest index wins ties.  The filter
+// is three packed max.bf16x2 on the raw words for bfloat16, three fmaxf for binary32.
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Monotone map from a float that is not NaN to a signed integer.
+__device__ __forceinline__ int float_order(float f) {
+    const int bits = __float_as_int(f);
+    return bits >= 0 ? bits : (bits ^ 0x7FFFFFFF);
+}
+__device__ __forceinline__ float float_unorder(int k) {
+    return __int_as_float(k >= 0 ? k : (k ^ 0x7FFFFFFF));
+}
+// The warp's largest st.best (no lane holds NaN there) and, for bfloat16, the packed pair
+// (f, f) with f the bfloat16 just below it, so that "greater than f" means ">= the maximum".
+__device__ __forceinline__ void refresh_floor(const RowState& st, float& floor_f, uint32_t& floor2) {
+    floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
+    int k = float_order(floor_f);
+    k -= 0x10000;  // one bfloat16 step down in the ordered domain (harmless below -inf)
+    const uint32_t hi = static_cast<uint32_t>(__float_as_int(float_unorder(k))) >> 16;
+    floor2 = floor_f == -INFINITY ? 0xFF80FF80u : (hi | (hi << 16));
+}
+template <int DT>
+__device__ __forceinline__ void track_best(const uint4& w, int first_index, float floor_f, uint32_t floor2,
+                                           RowState& st) {
+    constexpr int N = Elem<DT>::kPerVec;
+    if constexpr (DT == FEF_BF16) {
+        const uint32_t m = max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w));
+        if (floor_f != -INFINITY && max_bf16x2(floor2, m) == floor2) return;  // every element < the floor
+    }
+    float l[N];
+    unpack<DT>(w, l);
+    float vmax = l[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, l[i]);
+    if (vmax > st.best) {  // strict: an earlier (lower) index keeps a tie
+        int at = N - 1;
+#pragma unroll
+        for (int i = N - 2; i >= 0; --i)
+            if (l[i] == vmax) at = i;
+        st.best = vmax;
+        st.index = first_index + at;
+    }
+}
+
 template <bool GREEDY>
 __device__ __forceinline__ Partial warp_combine(float ref, float sum, float best, int index) {
     float M = ref;
@@ -386,17 +436,25 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 phase ^= 1u;
             }
             if (d.len > 0) {
+                if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
+                if (d.len == kTileBytes)  // branch-free: the four vectors interleave
+                    absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
+                else
+                    absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
                 if constexpr (GREEDY) {
+                    float floor_f;
+                    uint32_t floor2;
+                    refresh_floor(st, floor_f, floor2);
 #pragma unroll
                     for (int j = 0; j < kVecPerThread; ++j)
-                        if (at[j] < d.len)
-                            absorb_vector<DT, true>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, P.c_hi, P.c_lo, st);
-                } else {
-                    if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
-                    if (d.len == kTileBytes)  // branch-free: the four vectors interleave
-                        absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
-                    else
-                        absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
+                        if (at[j] < d.len) {
+                            if constexpr (DT == FEF_F32) {
+                                const float vmax = fmaxf(fmaxf(__uint_as_float(w[j].x), __uint_as_float(w[j].y)),
+                                                         fmaxf(__uint_as_float(w[j].z), __uint_as_float(w[j].w)));
+                                if (!(vmax >= floor_f)) continue;  // NaN never is the arg-max (the sum reports it)
+                            }
+                            track_best<DT>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, floor_f, floor2, st);
+                        }
                 }
             }
             if (d.flags & kFlagLast) {
@@ -641,6 +699,192 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
         P.tasks[b] = task;
     }
 }
+
+__device__ __forceinline__ double warp_max(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// The same as fold_unit, done by a whole warp: the lanes share the unit's partials.
+template <int DT, bool GREEDY>
+__device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const VerifyParams& P, int lane) {
+    const Geometry& G = P.geo;
+    const int nrec = G.claims_per_unit;
+    const Partial* rec = P.partials + u * G.claims_per_unit;
+    const int ntail = G.V - G.vec_elems;
+
+    // each lane folds its records into a running (m, s) pair, then the warp combines
+    double m = -INFINITY, sacc = 0.0;
+    int bad = 0;
+    float best = -INFINITY;
+    int index = 0x7FFFFFFF;
+    for (int r = lane; r < nrec; r += 32) {
+        const Partial p = rec[r];
+        if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = 1;
+        if (p.sum > 0.f) {
+            const double pm = p.ref, ps = p.sum;
+            if (pm > m) {
+                sacc = sacc * exp2(m - pm) + ps;
+                m = pm;
+            } else {
+                sacc += ps * exp2(pm - m);
+            }
+        }
+        if (GREEDY && better(p.best, p.index, best, index)) {
+            best = p.best;
+            index = p.index;
+        }
+    }
+    for (int j = lane; j < ntail; j += 32) {
+        const float l = load_logit<DT>(row, G.vec_elems + j);
+        if (l != l || l == INFINITY) {
+            bad = 1;
+        } else if (l > -INFINITY) {
+            const double pm = static_cast<double>(l) * c;
+            if (pm > m) {
+                sacc = sacc * exp2(m - pm) + 1.0;
+                m = pm;
+            } else {
+                sacc += exp2(pm - m);
+            }
+        }
+        if (GREEDY && better(l, G.vec_elems + j, best, index)) {
+            best = l;
+            index = G.vec_elems + j;
+        }
+    }
+    const double M = warp_max(m);
+    bad = __any_sync(0xFFFFFFFFu, bad);
+    if (GREEDY) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, index, o);
+            if (better(ob, oi, best, index)) {
+                best = ob;
+                index = oi;
+            }
+        }
+    }
+    const double S = warp_sum(m > -INFINITY ? sacc * exp2(m - M) : 0.0);
+    RowNorm out;
+    out.M = M;
+    out.S = S;
+    out.best = best;
+    out.index = index;
+    out.bad = bad || !(S > 0.0) || !(S < INFINITY);
+    return out;
+}
+
+constexpr int kScanMaxWarps = 32;
+
+// The same step with one CTA per window and one warp per position, for calls whose rows are
+// cut into many claims (few rows in all): the fold of a row's partials is then shared by 32 lanes.
+template <int DT, bool GREEDY>
+__global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __grid_constant__ VerifyParams P) {
+    const Geometry& G = P.geo;
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+    const int num_warps = blockDim.x >> 5;
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+
+    __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
+    __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
+    __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
+
+    for (int i = warp; i < n; i += num_warps) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + i;
+        const char* prow = P.target + row * G.ld_bytes;
+        const char* qrow = P.draft + row * G.ld_bytes;
+        const RowNorm np = fold_unit_warp<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P, lane);
+        RowNorm nq;
+        nq.bad = false;
+        if constexpr (!GREEDY) nq = fold_unit_warp<DT, false>(2 * row + 1, qrow, c, P, lane);
+        if (lane == 0) {
+            const int x = __ldg(P.draft_tokens + row);
+            int err = 0, accept = 0, alt = -1;
+            float conf = -1.f, conf_alt = -1.f;
+            double kp = 0.0, kq = 0.0;
+            if (x < 0 || x >= G.V) {
+                err = FEF_ERR_TOKEN_RANGE;
+            } else if (np.bad || nq.bad) {
+                err = FEF_ERR_NONFINITE;
+            } else {
+                kp = np.M + log2(np.S);
+                const double lpx = load_logit<DT>(prow, x);
+                const double l2pi = lpx * c - kp;  // log2 pi(x)
+                conf = static_cast<float>(exp2(l2pi));
+                if constexpr (GREEDY) {
+                    accept = (x == np.index);
+                    alt = np.index;
+                    conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
+                } else {
+                    kq = nq.M + log2(nq.S);
+                    const double lqx = load_logit<DT>(qrow, x);
+                    if (lqx == -INFINITY) {
+                        accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
+                    } else {
+                        const double ratio = exp2(l2pi - (lqx * c - kq));
+                        const uint4 r = philox4x32_10(
+                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), P.step),
+                            make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+                        const double uacc = uniform_from_word(r.x);
+                        accept = uacc <= fmin(1.0, ratio);
+                    }
+                }
+            }
+            s_err[i] = err;
+            s_accept[i] = accept;
+            s_conf[i] = conf;
+            s_conf_alt[i] = conf_alt;
+            s_alt[i] = alt;
+            s_kp[i] = kp;
+            s_kq[i] = kq;
+        }
+    }
+    __syncthreads();
+
+    int err = 0, a = n;
+    for (int i = 0; i < n; ++i) err = max(err, s_err[i]);
+    for (int i = n - 1; i >= 0; --i)
+        if (!s_accept[i]) a = i;
+
+    for (int i = threadIdx.x; i < G.K; i += blockDim.x) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + i;
+        int tok = -1;
+        float cf = -1.f;
+        if (!err) {
+            if (i < a) {
+                tok = __ldg(P.draft_tokens + row);
+                cf = s_conf[i];
+            } else if (GREEDY && i == a && a < n) {
+                tok = s_alt[i];
+                cf = s_conf_alt[i];
+            }
+        }
+        P.tokens[row] = tok;
+        P.conf[row] = cf;
+    }
+    if (threadIdx.x == 0) {
+        P.accept_len[b] = err ? -1 : a;
+        if (err) report(P.status, err);
+        ResidualTask task;
+        task.pos = (!GREEDY && !err && a < n) ? a : -1;
+        task.arrivals = 0u;
+        task.kp = task.pos >= 0 ? s_kp[a] : 0.0;
+        task.kq = task.pos >= 0 ? s_kq[a] : 0.0;
+        P.tasks[b] = task;
+    }
+}
+
 
 // ============================================================= residual ====
 constexpr int kResidualThreads = 256;
@@ -1032,8 +1276,13 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         g_attr_done[dev][which] = true;
     }
     stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, kSmemBytes, stream>>>(P);
-    cudaError_t e = launch_dependent(scan_kernel<DT, GREEDY>, dim3((G.B + kScanWarps - 1) / kScanWarps),
-                                     dim3(kScanWarps * 32), 0, stream, P);
+    cudaError_t e;
+    if (G.claims_per_unit >= 4)  // few rows, many partials per row: one warp per position
+        e = launch_dependent(scan_rows_kernel<DT, GREEDY>, dim3(G.B),
+                             dim3(32 * (G.K < kScanMaxWarps ? G.K : kScanMaxWarps)), 0, stream, P);
+    else
+        e = launch_dependent(scan_kernel<DT, GREEDY>, dim3((G.B + kScanWarps - 1) / kScanWarps), dim3(kScanWarps * 32),
+                             0, stream, P);
     if (e != cudaSuccess) return e;
     if (!GREEDY) {
         e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);

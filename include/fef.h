@@ -11,8 +11,8 @@
  * Conventions
  *  - Pointers marked "device" must be device memory of the current CUDA device;
  *    the caller owns every buffer.  The library allocates nothing, keeps no
- *    state between calls and never synchronises: all work (one kernel per call,
- *    preceded by the clearing of a few counters) is enqueued on `cuda_stream`
+ *    state between calls and never synchronises: all work (three kernels per
+ *    verification call, preceded by the clearing of a counter) is enqueued on `cuda_stream`
  *    (a cudaStream_t passed as void*; NULL = the default stream).
  *  - The return value reports what the host can see (bad arguments, launch
  *    failures).  Errors that only the data reveals are written to
@@ -113,6 +113,24 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
                            int32_t* accept_len, int32_t* tokens, float* conf,
                            void* workspace, size_t workspace_bytes,
                            int32_t* device_status, void* cuda_stream);
+
+/*
+ * fef_spec_verify with timing marks: the same operation (Algorithm 2's verification
+ * loop) and the same results, and additionally up to four caller-created CUDA events
+ * (cudaEvent_t passed as void*; NULL entries are skipped) are recorded on `cuda_stream`:
+ * [0] before the streaming kernel, [1] after it, [2] after the acceptance scan,
+ * [3] after the residual draw.  `stage_events` may be NULL.  Used to time the kernels
+ * separately; an event between two kernels keeps the later one from starting early, so
+ * the whole call is a little slower than fef_spec_verify.
+ */
+fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const int32_t* row_len,
+                                    int B, int K, int V, int64_t ld, fef_dtype dt,
+                                    float temperature, uint64_t seed, uint32_t step,
+                                    int32_t* accept_len, int32_t* tokens, float* conf,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* device_status, void* cuda_stream,
+                                    void* const* stage_events);
 
 /*
  * Host-buffer form of fef_spec_verify (same operation, same citations): every

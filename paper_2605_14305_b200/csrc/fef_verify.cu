@@ -1265,8 +1265,13 @@ static cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 blo
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+static void mark(void* const* events, int which, cudaStream_t stream) {
+    if (events && events[which]) cudaEventRecord(static_cast<cudaEvent_t>(events[which]), stream);
+}
+
+// events (may be null): [0] before the streaming kernel, [1] after it, [2] after the scan, [3] at the end
 template <int DT, bool GREEDY>
-static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream) {
+static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream, void* const* events) {
     const Geometry& G = P.geo;
     const int which = DT * 2 + (GREEDY ? 1 : 0);
     if (!g_attr_done[dev][which]) {
@@ -1275,7 +1280,9 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         if (e != cudaSuccess) return e;
         g_attr_done[dev][which] = true;
     }
+    mark(events, 0, stream);
     stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, kSmemBytes, stream>>>(P);
+    mark(events, 1, stream);
     cudaError_t e;
     if (G.claims_per_unit >= 4)  // few rows, many partials per row: one warp per position
         e = launch_dependent(scan_rows_kernel<DT, GREEDY>, dim3(G.B),
@@ -1284,10 +1291,12 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         e = launch_dependent(scan_kernel<DT, GREEDY>, dim3((G.B + kScanWarps - 1) / kScanWarps), dim3(kScanWarps * 32),
                              0, stream, P);
     if (e != cudaSuccess) return e;
+    mark(events, 2, stream);
     if (!GREEDY) {
         e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
         if (e != cudaSuccess) return e;
     }
+    mark(events, 3, stream);
     return cudaGetLastError();
 }
 
@@ -1320,11 +1329,12 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
     return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
 }
 
-fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
-                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
-                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
-                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
-                           int32_t* device_status, void* cuda_stream) {
+fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
+                                    int64_t ld, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
+                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
+                                    void* const* stage_events) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -1386,10 +1396,22 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, 
     if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return FEF_ERR_CUDA;
     cudaError_t e;
     if (dt == FEF_F32)
-        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream) : launch_all<FEF_F32, false>(P, dev, stream);
+        e = greedy ? launch_all<FEF_F32, true>(P, dev, stream, stage_events)
+                   : launch_all<FEF_F32, false>(P, dev, stream, stage_events);
     else
-        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream) : launch_all<FEF_BF16, false>(P, dev, stream);
+        e = greedy ? launch_all<FEF_BF16, true>(P, dev, stream, stage_events)
+                   : launch_all<FEF_BF16, false>(P, dev, stream, stage_events);
     return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* cuda_stream) {
+    return fef_spec_verify_profiled(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt,
+                                    temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes,
+                                    device_status, cuda_stream, nullptr);
 }
 
 // ---- host-buffer variant: layout of the caller's device arena

@@ -328,6 +328,19 @@ def test_host_buffer_entry_points_match_device_entry_points(fef):
     assert err.value.status == fef.FEF_ERR_WORKSPACE
 
 
+def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef):
+    q, p, tok = _random_case(4, 16, 50000, torch.bfloat16, 0.7, 51)
+    want = _gpu_verify(fef, q, p, tok, 1.0, 3, 3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for e in ev:
+        e.record()
+    r = fef.fef_spec_verify(q, p, tok, 1.0, 3, 3, stage_events=ev)
+    torch.cuda.synchronize()
+    assert (r.accept_len.cpu().numpy() == want[0]).all() and (r.tokens.cpu().numpy() == want[1]).all()
+    assert (r.conf.cpu().numpy() == want[2]).all()
+    assert all(ev[i].elapsed_time(ev[i + 1]) > 0 for i in range(3))
+
+
 def test_api_errors_with_real_buffers(fef):
     q, p, tok = _random_case(2, 4, 64, torch.float32, 0.5, 61)
     lib = fef.load()

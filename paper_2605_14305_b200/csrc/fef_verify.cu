@@ -176,9 +176,10 @@ __device__ __forceinline__ float first_reference(const uint4& w, float c_hi, flo
 // A thread's share of one tile in sampling mode: the vectors with offset < len, one
 // overflow check for the whole tile.  When the check fires (reference far too low or
 // missing, or bad data) the tile is redone vector by vector through absorb_vector,
-// which moves the reference.
+// which moves the reference.  Returns the thread's sum over the tile relative to st.ref, or
+// NaN when the tile went the slow way.
 template <int DT, bool FULL>
-__device__ __forceinline__ void absorb_tile(const uint4 (&w)[kVecPerThread], const int (&at)[kVecPerThread], int len,
+__device__ __forceinline__ float absorb_tile(const uint4 (&w)[kVecPerThread], const int (&at)[kVecPerThread], int len,
                                             float c_hi, float c_lo, RowState& st) {
     const float2 ch = make_float2(c_hi, c_hi);
     const float2 cl = make_float2(c_lo, c_lo);
@@ -191,50 +192,32 @@ __device__ __forceinline__ void absorb_tile(const uint4 (&w)[kVecPerThread], con
     const float ts = acc.x + acc.y;
     if (ts <= kRescaleAbove) {
         st.sum += ts;
-    } else {
-#pragma unroll
-        for (int j = 0; j < kVecPerThread; ++j)
-            if (FULL || at[j] < len) absorb_vector<DT, false>(w[j], 0, c_hi, c_lo, st);
+        return ts;
     }
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j)
+        if (FULL || at[j] < len) absorb_vector<DT, false>(w[j], 0, c_hi, c_lo, st);
+    return __int_as_float(0x7FC00000);
 }
 
 // Butterfly over the warp: every lane ends with the combination of all 32 records
 // (same tree in every lane, so the result does not depend on who asks).
-// Greedy mode: largest logit of the thread's share and its lowest index.  The exact update
-// (unpack, compare, find the index) runs only for a vector that holds an element >= the warp's
-// running maximum (refreshed once per tile); anything smaller cannot be the row's arg-max, and
-// equal elements still go through the exact update, so the lowest index wins ties.  The filter
-// is three packed max.bf16x2 on the raw words for bfloat16, three fmaxf for binary32.
-__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
-// Monotone map from a float that is not NaN to a signed integer.
-__device__ __forceinline__ int float_order(float f) {
+// Greedy mode: largest logit of the thread's share and its lowest index.  The exact update below
+// (unpack, compare, find the index) runs only for tiles that can hold a new maximum: a thread's
+// tile sum of 2^(l c - ref), which the streaming pass computes anyway, is at least the largest
+// of its terms, so a sum below 2^(floor c - ref) rules the whole tile out.  The floor is the
+// warp's running maximum (refreshed once per tile); an element equal to it in a later tile has a
+// higher index than its holder, so it need not be looked at.
+__device__ __forceinline__ int float_order(float f) {  // monotone map, floats without NaN -> int
     const int bits = __float_as_int(f);
     return bits >= 0 ? bits : (bits ^ 0x7FFFFFFF);
 }
 __device__ __forceinline__ float float_unorder(int k) {
     return __int_as_float(k >= 0 ? k : (k ^ 0x7FFFFFFF));
 }
-// The warp's largest st.best (no lane holds NaN there) and, for bfloat16, the packed pair
-// (f, f) with f the bfloat16 just below it, so that "greater than f" means ">= the maximum".
-__device__ __forceinline__ void refresh_floor(const RowState& st, float& floor_f, uint32_t& floor2) {
-    floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
-    int k = float_order(floor_f);
-    k -= 0x10000;  // one bfloat16 step down in the ordered domain (harmless below -inf)
-    const uint32_t hi = static_cast<uint32_t>(__float_as_int(float_unorder(k))) >> 16;
-    floor2 = floor_f == -INFINITY ? 0xFF80FF80u : (hi | (hi << 16));
-}
 template <int DT>
-__device__ __forceinline__ void track_best(const uint4& w, int first_index, float floor_f, uint32_t floor2,
-                                           RowState& st) {
+__device__ __forceinline__ void track_best(const uint4& w, int first_index, RowState& st) {
     constexpr int N = Elem<DT>::kPerVec;
-    if constexpr (DT == FEF_BF16) {
-        const uint32_t m = max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w));
-        if (floor_f != -INFINITY && max_bf16x2(floor2, m) == floor2) return;  // every element < the floor
-    }
     float l[N];
     unpack<DT>(w, l);
     float vmax = l[0];
@@ -437,24 +420,23 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             }
             if (d.len > 0) {
                 if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
+                float tile_sum;
                 if (d.len == kTileBytes)  // branch-free: the four vectors interleave
-                    absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
+                    tile_sum = absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
                 else
-                    absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
+                    tile_sum = absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
                 if constexpr (GREEDY) {
-                    float floor_f;
-                    uint32_t floor2;
-                    refresh_floor(st, floor_f, floor2);
+                    const float floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
+                    // 0.999: the sum and the bound carry a few units of 1e-7 of rounding each
+                    const bool candidate = !(tile_sum < 0.999f * exp2_scaled<DT>(floor_f, P.c_hi, P.c_lo, st.ref));
+                    if (__any_sync(0xFFFFFFFFu, candidate)) {  // the vote keeps this out of the straight-line code
+                        if (candidate) {
 #pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j)
-                        if (at[j] < d.len) {
-                            if constexpr (DT == FEF_F32) {
-                                const float vmax = fmaxf(fmaxf(__uint_as_float(w[j].x), __uint_as_float(w[j].y)),
-                                                         fmaxf(__uint_as_float(w[j].z), __uint_as_float(w[j].w)));
-                                if (!(vmax >= floor_f)) continue;  // NaN never is the arg-max (the sum reports it)
-                            }
-                            track_best<DT>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, floor_f, floor2, st);
+                            for (int j = 0; j < kVecPerThread; ++j)
+                                if (at[j] < d.len)
+                                    track_best<DT>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, st);
                         }
+                    }
                 }
             }
             if (d.flags & kFlagLast) {

@@ -962,7 +962,7 @@ __device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kResidualThreads, 3) residual_kernel(const __grid_constant__ VerifyParams P) {
+__global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __grid_constant__ VerifyParams P) {
     constexpr int N = Elem<DT>::kPerVec;
     const Geometry& G = P.geo;
     cudaGridDependencySynchronize();  // the scan kernel's tasks must be complete and visible
@@ -1204,6 +1204,10 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool gr
            static_cast<int64_t>(B) * ((nvec + kResidualThreads * per_thread - 1) / (kResidualThreads * per_thread)) < 2 * sm_count)
         per_thread >>= 1;
     int parts = (nvec + kResidualThreads * per_thread - 1) / (kResidualThreads * per_thread);
+    // all CTAs of the call resident at once (four per SM) where that is possible: one wave of
+    // CTAs that loop beats several waves of CTAs that each pay the start-up latencies
+    const int resident = (4 * sm_count) / B;
+    if (resident >= 1 && parts > resident) parts = resident;
     if (parts > kMaxResidualCtas) parts = kMaxResidualCtas;
     if (parts < 1) parts = 1;
     G.residual_ctas = parts;

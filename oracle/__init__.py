@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
                 vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, u32, vp, vp, vp, vp, vp,
             ]
             L.fef_oracle_spec_verify.restype = i32
+            L.fef_oracle_draft_sample.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, u32, vp, vp]
+            L.fef_oracle_draft_sample.restype = i32
             L.fef_oracle_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp]
             L.fef_oracle_remask_select.restype = i32
             _lib = L
@@ -156,6 +158,23 @@ def spec_verify(draft_logits, target_logits, draft_tokens, temperature, seed, st
         _ptr(accept_len), _ptr(tokens), _ptr(conf), _ptr(margin), _ptr(gap),
     )
     return dict(status=st, accept_len=accept_len, tokens=tokens, conf=conf, accept_margin=margin, gumbel_gap=gap)
+
+
+def draft_sample(draft_logits, temperature, seed, step, row_len=None, V=None, batch_offset=0):
+    """Draw the draft tokens of one call.  Logits are [B, K, ld]; ``V`` defaults to ld.
+
+    Returns a dict: status, tokens [B,K] (int32, -1 where nothing was drawn), gumbel_gap [B,K].
+    """
+    q, dt = _logits_as_numpy(draft_logits)
+    assert q.ndim == 3
+    B, K, ld = q.shape
+    V = ld if V is None else V
+    rl = None if row_len is None else _i32(row_len).reshape(B)
+    tokens = np.zeros((B, K), dtype=np.int32)
+    gap = np.zeros((B, K), dtype=np.float64)
+    st = lib().fef_oracle_draft_sample(_ptr(q), _ptr(rl), B, K, V, ld, dt, temperature, seed, step, batch_offset,
+                                       _ptr(tokens), _ptr(gap))
+    return dict(status=st, tokens=tokens, gumbel_gap=gap)
 
 
 def remask_select(conf, mask, k):

@@ -128,6 +128,7 @@ double uniform_open01(uint64_t seed, uint32_t stream, uint32_t j, uint32_t b, ui
 
 const uint32_t kStreamAccept = 0;    // one uniform per (b, pos, step)
 const uint32_t kStreamResidual = 1;  // one uniform per (b, pos, step, vocabulary id)
+const uint32_t kStreamDraft = 2;     // draft sampling: one uniform per (b, pos, step, vocabulary id)
 
 // -------------------------------------------------------------- residual ----
 // r_x = [pi(x) - rho(x)]_+   (numerator of the residual law)
@@ -254,6 +255,45 @@ int verify_one_window(const void* q_base, const void* p_base, const int32_t* dra
     return FEFO_OK;
 }
 
+// ---------------------------------------------------------- draft sampling ----
+// x~ ~ softmax(l / T) for one position (Algorithm 2, "Sample draft tokens"; Section 3.2) by
+// Gumbel-max: arg-max over x of l_x / T - ln(-ln u_x), one uniform per vocabulary id, entries
+// with l_x = -inf left out, lowest x on exact ties.  T == 0: arg-max of l (lowest index).
+// Returns the token, -1 on a data error (NaN, +inf, or no finite logit).  *gap = best score
+// minus runner-up score (in units of l / T; +inf with a single candidate or at T == 0).
+int sample_draft_row(const void* row, int V, int dtype, double T, uint64_t seed, uint32_t b, uint32_t pos,
+                     uint32_t step, double* gap, int* status) {
+    int best = -1;
+    double best_score = -kInf, second_score = -kInf;
+    *gap = kInf;
+    for (int x = 0; x < V; ++x) {
+        const double l = load_logit(row, x, dtype);
+        if (std::isnan(l) || l == kInf) {
+            *status = FEFO_ERR_NONFINITE;
+            return -1;
+        }
+        if (l == -kInf) continue;
+        double score = l;
+        if (T > 0.0) {
+            const double u = uniform_open01(seed, kStreamDraft, (uint32_t)x >> 2, b, pos, step, (uint32_t)x & 3u);
+            score = l / T - std::log(-std::log(u));
+        }
+        if (score > best_score) {  // strict: the lowest x keeps an exact tie
+            second_score = best_score;
+            best_score = score;
+            best = x;
+        } else if (score > second_score) {
+            second_score = score;
+        }
+    }
+    if (best < 0) {
+        *status = FEFO_ERR_NONFINITE;
+        return -1;
+    }
+    if (T > 0.0 && second_score > -kInf) *gap = best_score - second_score;
+    return best;
+}
+
 }  // namespace
 
 // ================================================================= C ABI ====
@@ -345,6 +385,33 @@ int fef_oracle_remask_select(const float* conf, const uint8_t* mask, int B, int 
         for (int t = 0; t < k; ++t) positions[(int64_t)b * k + t] = t < n ? cand[(size_t)t] : -1;
     }
     return FEFO_OK;
+}
+
+int fef_oracle_draft_sample(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
+                            int dtype, float temperature, uint64_t seed, uint32_t step, uint32_t batch_offset,
+                            int32_t* draft_tokens, double* gumbel_gap) {
+    if (!draft_logits || !draft_tokens || B < 1 || K < 1 || V < 1 || ld < V) return FEFO_ERR_INVALID_ARG;
+    if (dtype != FEFO_F32 && dtype != FEFO_BF16) return FEFO_ERR_DTYPE;
+    if (!(temperature >= 0.0f)) return FEFO_ERR_INVALID_ARG;
+    const int64_t esize = dtype == FEFO_F32 ? 4 : 2;
+    int worst = FEFO_OK;
+    for (int b = 0; b < B; ++b) {
+        const int n = row_len ? std::min(std::max(row_len[b], 0), K) : K;
+        for (int i = 0; i < K; ++i) {
+            const int64_t row = (int64_t)b * K + i;
+            draft_tokens[row] = -1;
+            if (gumbel_gap) gumbel_gap[row] = kInf;
+            if (i >= n) continue;
+            int status = FEFO_OK;
+            double gap = kInf;
+            const char* base = (const char*)draft_logits + row * ld * esize;
+            draft_tokens[row] = sample_draft_row(base, V, dtype, (double)temperature, seed, batch_offset + (uint32_t)b,
+                                                 (uint32_t)i, step, &gap, &status);
+            if (gumbel_gap) gumbel_gap[row] = gap;
+            worst = std::max(worst, status);
+        }
+    }
+    return worst;
 }
 
 }  // extern "C"

@@ -17,7 +17,8 @@
  * = sum_z min(pi, rho), emitted-token law = pi by exact enumeration and by
  * chi-square, p = q accepts everything, residual sums to one, mean committed
  * length = sum_l prod_{i<l} alpha_i (Theorem 2 when the alpha_i are equal),
- * LowConf against a library stable sort.
+ * LowConf against a library stable sort; draft sampling: frequencies against a library softmax
+ * by chi-square, the temperature-0 limit against arg-max, invariance under a common shift.
  * Parity unpinned by the paper (readings fixed by this build only): the
  * confidence reported at temperature 0, tie order in LowConf, sentinel values
  * beyond the committed prefix.
@@ -86,6 +87,18 @@ int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
                            uint32_t batch_offset,
                            int32_t* accept_len, int32_t* tokens, double* conf,
                            double* accept_margin, double* gumbel_gap);
+
+/* Draft-token sampling (Algorithm 2, "Sample draft tokens x~ ~ rho"; Section 3.2): for every
+ * position i < row_len[b] one draw from rho = softmax(draft_logits[b,i,:] / T) by Gumbel-max,
+ * arg-max_x { l_x / T - ln(-ln u_x) } over the entries with l_x > -inf, lowest x on exact ties;
+ * u_x from stream 2: counter ((2 << 30) | (x >> 2), batch_offset + b, i, step), word x & 3.
+ * T == 0: arg-max of the logits, no random numbers.
+ *   draft_tokens [B, K]  the draws; -1 for i >= row_len[b] and for positions with a data error
+ *   gumbel_gap   [B, K]  (may be NULL) best minus runner-up score, +inf if there is none
+ * Returns the largest status (NaN, +inf or a row without a finite logit: FEFO_ERR_NONFINITE). */
+int fef_oracle_draft_sample(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
+                            int dtype, float temperature, uint64_t seed, uint32_t step, uint32_t batch_offset,
+                            int32_t* draft_tokens, double* gumbel_gap);
 
 /* LowConf_k (Algorithm 2): per batch row the k candidates (mask != 0) of lowest
  * confidence, ordered by (conf ascending, index ascending).

@@ -531,3 +531,84 @@ def test_remask_select_brute_force_all_tie_patterns():
             cand = sorted((pattern[i], i) for i in range(L) if mask[0, i])
             want = [i for _, i in cand][:k]
             assert cnt[0] == len(want) and pos[0, :len(want)].tolist() == want
+
+
+# ----------------------------------------------------------- draft sampling ----
+# Algorithm 2, "Sample draft tokens x~ ~ rho"; Section 3.2.  The oracle draws by Gumbel-max;
+# what pins it is the law it must produce (a library softmax), not its own arithmetic.
+@pytest.mark.parametrize("V,T", [(4, 1.0), (16, 0.7), (11, 2.5)])
+def test_draft_sample_frequencies_match_library_softmax_chi_square(V, T):
+    rng = np.random.default_rng(100 + V)
+    logits = rng.normal(0.0, 1.5, size=V).astype(np.float32)
+    n = 60000
+    # n independent draws: one position per batch row, so every draw has its own counter
+    out = oracle.draft_sample(_tile(logits, n), T, seed=4242, step=3)
+    assert out["status"] == 0
+    counts = np.bincount(out["tokens"].ravel(), minlength=V)
+    expected = _softmax64(logits, T) * n
+    chi2 = ((counts - expected) ** 2 / expected).sum()
+    assert chi2 < stats.chi2.ppf(0.9999, V - 1), (chi2, counts, expected)
+
+
+def test_draft_sample_positions_steps_and_seeds_draw_independently():
+    # uniform law over 8 ids, 64 windows of 8 positions: every change of the stream must show
+    logits = _f32(np.zeros((64, 8, 8), dtype=np.float32))
+    a = oracle.draft_sample(logits, 1.0, seed=1, step=0)["tokens"]
+    assert len({tuple(r) for r in a}) > 60                         # batch rows differ
+    assert (a[:, 0] != a[:, 1]).mean() > 0.7                       # positions differ
+    assert (oracle.draft_sample(logits, 1.0, seed=1, step=1)["tokens"] != a).mean() > 0.7
+    assert (oracle.draft_sample(logits, 1.0, seed=2, step=0)["tokens"] != a).mean() > 0.7
+    # a slice of the batch drawn on its own, with its offset, repeats the full batch's draws
+    b = oracle.draft_sample(logits[:10], 1.0, seed=1, step=0, batch_offset=20)["tokens"]
+    assert (b == a[20:30]).all()
+    # and the stream is not the one the verification step uses for its residual draw
+    u_draft = oracle.uniform(1, 2, 0, 0, 0, 0, 0)
+    assert u_draft != oracle.uniform(1, 1, 0, 0, 0, 0, 0) and u_draft != oracle.uniform(1, 0, 0, 0, 0, 0, 0)
+
+
+def test_draft_sample_uses_one_uniform_per_vocabulary_id_as_documented():
+    # brute force from the documented recipe: u_x = uniform(seed, stream 2, x >> 2, b, i, step, x & 3)
+    rng = np.random.default_rng(5)
+    B, K, V, T = 3, 2, 37, 0.8
+    logits = rng.normal(0, 2, size=(B, K, V)).astype(np.float32)
+    out = oracle.draft_sample(_f32(logits), T, seed=77, step=9)
+    for b in range(B):
+        for i in range(K):
+            u = np.array([oracle.uniform(77, 2, x >> 2, b, i, 9, x & 3) for x in range(V)])
+            scores = logits[b, i].astype(np.float64) / T - np.log(-np.log(u))
+            assert out["tokens"][b, i] == int(np.argmax(scores))
+            top2 = np.sort(scores)[-2:]
+            assert abs(out["gumbel_gap"][b, i] - (top2[1] - top2[0])) < 1e-9
+
+
+def test_draft_sample_shift_invariance_low_temperature_and_greedy():
+    rng = np.random.default_rng(6)
+    logits = rng.normal(0, 2, size=(5, 4, 50)).astype(np.float32)
+    base = oracle.draft_sample(_f32(logits), 1.3, seed=3, step=1)["tokens"]
+    # a common offset per row does not change a softmax law, nor the draw (the offset is exact in binary32)
+    assert (oracle.draft_sample(_f32(logits + 64.0), 1.3, seed=3, step=1)["tokens"] == base).all()
+    amax = logits.argmax(-1)
+    assert (oracle.draft_sample(_f32(logits), 0.0, seed=3, step=1)["tokens"] == amax).all()
+    assert (oracle.draft_sample(_f32(logits), 1e-4, seed=3, step=1)["tokens"] == amax).all()
+    # ties at temperature 0: lowest index
+    tied = np.zeros((1, 1, 9), dtype=np.float32)
+    tied[0, 0, [3, 7]] = 2.0
+    assert oracle.draft_sample(_f32(tied), 0.0, seed=0, step=0)["tokens"][0, 0] == 3
+
+
+def test_draft_sample_zero_probability_entries_row_len_and_errors():
+    logits = np.zeros((2, 3, 6), dtype=np.float32)
+    logits[:, :, [0, 2, 5]] = -np.inf
+    out = oracle.draft_sample(_f32(np.repeat(logits, 200, axis=0)), 1.0, seed=8, step=0)
+    assert set(np.unique(out["tokens"])) == {1, 3, 4}              # -inf entries are never drawn
+    rl = np.array([2, 0], dtype=np.int32)
+    out = oracle.draft_sample(_f32(logits), 1.0, seed=8, step=0, row_len=rl)
+    assert (out["tokens"][0, :2] >= 0).all() and (out["tokens"][0, 2:] == -1).all() and (out["tokens"][1] == -1).all()
+    bad = np.zeros((3, 1, 4), dtype=np.float32)
+    bad[0, 0, 1] = np.nan
+    bad[1, 0, :] = -np.inf
+    out = oracle.draft_sample(_f32(bad), 1.0, seed=8, step=0)
+    assert out["status"] == oracle.ERR_NONFINITE
+    assert out["tokens"][0, 0] == -1 and out["tokens"][1, 0] == -1 and out["tokens"][2, 0] >= 0
+    bf = torch.tensor(np.random.default_rng(1).normal(0, 2, size=(4, 2, 33)).astype(np.float32)).to(torch.bfloat16)
+    assert (oracle.draft_sample(bf, 0.9, 5, 5)["tokens"] == oracle.draft_sample(bf.float(), 0.9, 5, 5)["tokens"]).all()

@@ -575,7 +575,7 @@ def test_draft_sample_uses_one_uniform_per_vocabulary_id_as_documented():
     for b in range(B):
         for i in range(K):
             u = np.array([oracle.uniform(77, 2, x >> 2, b, i, 9, x & 3) for x in range(V)])
-            scores = logits[b, i].astype(np.float64) / T - np.log(-np.log(u))
+            scores = logits[b, i].astype(np.float64) / float(np.float32(T)) - np.log(-np.log(u))  # T is a binary32 argument
             assert out["tokens"][b, i] == int(np.argmax(scores))
             top2 = np.sort(scores)[-2:]
             assert abs(out["gumbel_gap"][b, i] - (top2[1] - top2[0])) < 1e-9

@@ -189,6 +189,39 @@ fef_status fef_spec_verify_static(const void* draft_logits, const void* target_l
                                   int32_t* device_status, void* cuda_stream);
 
 /*
+ * Draft-token sampling (Algorithm 2, "Sample draft tokens x~ ~ rho"; Section 3.2, "We then
+ * sample draft tokens ..."): for every window b and position i < n_b one draw
+ *   draft_tokens[b,i] ~ rho_i = softmax(draft_logits[b,i,:] / T),
+ * taken by Gumbel-max: arg-max over x of l_x / T - ln(-ln u_x) among the entries with
+ * l_x > -inf, lowest x on exact ties.  u_x comes from Philox4x32-10 keyed like fef_spec_verify,
+ * stream 2: counter ((2 << 30) | (x >> 2), b, i, step), output word x & 3,
+ * u = ((r >> 9) + 0.5) * 2^-23.  Temperature 0: arg-max of the logits (lowest index on ties),
+ * no random numbers.  Pass the same `seed` and `step` as to the fef_spec_verify call that
+ * checks these drafts: the two calls use different Philox streams.
+ *
+ * Arguments
+ *   draft_logits   device, [B, K, ld] row-major, dtype `dt`, same layout and alignment rules as
+ *                  fef_spec_verify; -inf entries are legal (never drawn)
+ *   row_len        device, [B] int32 in [0, K], or NULL = K everywhere
+ *   draft_tokens   device out, [B, K] int32; -1 for i >= n_b and for positions with a data error
+ *   log2_norm      device out, [B, K] float64, or NULL: log2 of sum_x 2^(l_x * log2(e) / T), the
+ *                  normaliser of rho_i (rho_i(x) = 2^(l_x log2(e) / T - log2_norm)); at T = 0 the
+ *                  T = 1 value; 0 where no token was drawn
+ *   workspace      device scratch of at least fef_draft_sample_workspace_bytes(...) bytes,
+ *                  256-byte aligned, contents need not be initialised
+ *   device_status  device out, [1] int32, or NULL: FEF_OK, or FEF_ERR_NONFINITE when a used row
+ *                  holds NaN or +inf or no finite logit (that position gets token -1)
+ * Asynchronous on `cuda_stream`; one kernel.
+ */
+size_t fef_draft_sample_workspace_bytes(int B, int K, int V, fef_dtype dt);
+fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len,
+                            int B, int K, int V, int64_t ld, fef_dtype dt,
+                            float temperature, uint64_t seed, uint32_t step,
+                            int32_t* draft_tokens, double* log2_norm,
+                            void* workspace, size_t workspace_bytes,
+                            int32_t* device_status, void* cuda_stream);
+
+/*
  * LowConf_k of Algorithm 2 ("Select R = LowConf_{n_rm}(C)"): for every batch
  * row the k candidate positions of lowest confidence.
  *

@@ -24,7 +24,8 @@ FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
 
 EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_spec_verify_profiled",
            "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
-           "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static")
+           "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static",
+           "fef_draft_sample_workspace_bytes", "fef_draft_sample")
 
 _lib = None
 
@@ -64,6 +65,10 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_host.restype = i32
     L.fef_spec_verify_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp]
     L.fef_spec_verify_static.restype = i32
+    L.fef_draft_sample_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.fef_draft_sample_workspace_bytes.restype = sz
+    L.fef_draft_sample.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, sz, vp, vp]
+    L.fef_draft_sample.restype = i32
     L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.fef_remask_select.restype = i32
     L.fef_remask_select_host_arena_bytes.argtypes = [i32, i32, i32]
@@ -158,6 +163,53 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
             st = load().fef_spec_verify_profiled(*args, handles)
     if st != FEF_OK:
         raise FefError(st, "fef_spec_verify")
+    return out
+
+
+class DraftResult(NamedTuple):
+    tokens: torch.Tensor         # [B, K] int32, -1 where nothing was drawn
+    log2_norm: torch.Tensor      # [B, K] float64
+    device_status: torch.Tensor  # [1] int32 (read it after synchronising)
+
+
+def fef_draft_sample_workspace_bytes(B: int, K: int, V: int, dtype) -> int:
+    code = dtype if isinstance(dtype, int) else (FEF_F32 if dtype == torch.float32 else FEF_BF16)
+    return int(load().fef_draft_sample_workspace_bytes(B, K, V, code))
+
+
+def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, step: int,
+                     row_len: Optional[torch.Tensor] = None, V: Optional[int] = None,
+                     out: Optional[DraftResult] = None, workspace: Optional[torch.Tensor] = None,
+                     stream=None) -> DraftResult:
+    """Enqueue the draft-token draws of one call (see ``fef_draft_sample`` in include/fef.h).
+
+    ``draft_logits``: ``[B, K, ld]`` CUDA tensor, float32 or bfloat16, contiguous; ``V`` (default
+    ``ld``) entries of each row are used.  Asynchronous on the current (or given) stream.
+    """
+    _require_cuda(draft_logits, row_len)
+    if draft_logits.dim() != 3 or not draft_logits.is_contiguous():
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_draft_sample")
+    if row_len is not None and row_len.dtype != torch.int32:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_draft_sample")
+    B, K, ld = draft_logits.shape
+    V = ld if V is None else int(V)
+    code = _dtype_code(draft_logits)
+    dev = draft_logits.device
+    with torch.cuda.device(dev):
+        if out is None:
+            out = DraftResult(torch.empty((B, K), dtype=torch.int32, device=dev),
+                              torch.empty((B, K), dtype=torch.float64, device=dev),
+                              torch.empty(1, dtype=torch.int32, device=dev))
+        if workspace is None:
+            workspace = torch.empty(max(fef_draft_sample_workspace_bytes(B, K, V, code), 256), dtype=torch.uint8,
+                                    device=dev)
+        st = load().fef_draft_sample(draft_logits.data_ptr(), None if row_len is None else row_len.data_ptr(),
+                                     B, K, V, ld, code, float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                     int(step) & 0xFFFFFFFF, out.tokens.data_ptr(), out.log2_norm.data_ptr(),
+                                     workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(),
+                                     _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_draft_sample")
     return out
 
 
@@ -296,6 +348,6 @@ def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena
     return positions, count
 
 
-__all__ = ["fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
+__all__ = ["fef_draft_sample", "fef_draft_sample_workspace_bytes", "DraftResult", "fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]

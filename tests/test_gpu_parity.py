@@ -363,3 +363,77 @@ def test_api_errors_with_real_buffers(fef):
     torch.cuda.synchronize()
     assert fef.fef_spec_verify_workspace_bytes(2, 4, 64, torch.float32) > 0
     assert fef.fef_spec_verify_workspace_bytes(2, 65, 64, torch.float32) == 0
+
+
+# ------------------------------------------------------------ draft sampling ----
+def _check_draft(fef, q, T, seed, step, row_len=None, V=None, expect_status=0):
+    """fef_draft_sample against the oracle on the same bytes: tokens exact, except positions whose
+    two best Gumbel scores lie within 1e-6 of each other (counted, must stay rare); normaliser to 1e-6."""
+    r = fef.fef_draft_sample(q, T, seed, step, row_len=row_len, V=V)
+    torch.cuda.synchronize()
+    ref = oracle.draft_sample(q.cpu(), T, seed, step, row_len=None if row_len is None else row_len.cpu(), V=V)
+    assert ref["status"] == expect_status and int(r.device_status.item()) == expect_status
+    got = r.tokens.cpu().numpy()
+    differ = got != ref["tokens"]
+    excused = differ & (ref["gumbel_gap"] < 1e-6)
+    assert not (differ & ~excused).any(), (np.argwhere(differ & ~excused)[:5], got[differ][:5], ref["tokens"][differ][:5])
+    drawn = ref["tokens"] >= 0
+    if drawn.any():
+        Vv = q.shape[-1] if V is None else V
+        Tn = T if T > 0 else 1.0
+        want = torch.logsumexp(q.cpu()[..., :Vv].double() / float(np.float32(Tn)), dim=-1).numpy() / math.log(2.0)
+        assert np.allclose(r.log2_norm.cpu().numpy()[drawn], want[drawn], rtol=0, atol=2e-5)
+    return int(excused.sum()), int(drawn.sum())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T", [1.0, 0.7, 0.0])
+def test_draft_sample_small_shapes_match_oracle(fef, dtype, T):
+    excused = drawn = 0
+    for n, (B, K, V, ld) in enumerate(SMALL_SHAPES):
+        if dtype == torch.bfloat16:
+            ld = (ld + 7) // 8 * 8
+        q, _, _ = _random_case(B, K, V, dtype, 0.8, 300 + n, ld=ld)
+        e, d = _check_draft(fef, q, T, seed=11 + n, step=n, V=V)
+        excused += e
+        drawn += d
+    assert excused <= 1 and drawn > 1000
+
+
+def test_draft_sample_llada_and_dream_shapes_row_len_and_errors(fef):
+    w = synth.LLADA_BATCHED.with_(B=4, K=8)
+    q, _ = synth.make_logits(w, seed=5, device="cuda")
+    assert _check_draft(fef, q, 0.7, 21, 1)[0] == 0
+    rl = torch.tensor([8, 0, 3, 1], dtype=torch.int32, device="cuda")
+    assert _check_draft(fef, q, 1.0, 21, 2, row_len=rl)[0] == 0
+    wd = synth.DREAM_LARGE.with_(B=2, K=4)
+    qd, _ = synth.make_logits(wd, seed=6, device="cuda")
+    assert _check_draft(fef, qd, 1.0, 22, 3)[0] == 0
+    assert _check_draft(fef, qd, 0.0, 22, 4)[0] == 0
+    # one draw per row of a single window: the row is shared by many CTAs
+    ws = synth.LLADA_SINGLE.with_(K=3)
+    qs, _ = synth.make_logits(ws, seed=7, device="cuda")
+    assert _check_draft(fef, qs, 1.0, 23, 5)[0] == 0
+    # -inf entries are never drawn; NaN, +inf and a row without a finite logit are data errors
+    qe = q.clone()
+    qe[0, 0, ::2] = float("-inf")
+    assert _check_draft(fef, qe, 1.0, 24, 6)[0] == 0
+    qe[1, 2, 77] = float("nan")
+    qe[2, 1, :] = float("-inf")
+    qe[3, 0, 5] = float("inf")
+    _check_draft(fef, qe, 1.0, 24, 7, expect_status=fef.FEF_ERR_NONFINITE)
+    # the same call twice gives the same tokens (no race in the reductions)
+    a = fef.fef_draft_sample(q, 0.9, 1, 1).tokens.clone()
+    b = fef.fef_draft_sample(q, 0.9, 1, 1).tokens
+    torch.cuda.synchronize()
+    assert (a == b).all()
+
+
+def test_draft_tokens_feed_verification(fef):
+    """Drafts drawn on the device go straight into fef_spec_verify; the pair matches the oracle pair."""
+    w = synth.LLADA_BATCHED.with_(B=3, K=16)
+    q, p = synth.make_logits(w, seed=9, device="cuda")
+    d = fef.fef_draft_sample(q, 0.7, 31, 4)
+    _check(fef, q, p, d.tokens, 0.7, 31, 4)
+    od = oracle.draft_sample(q.cpu(), 0.7, 31, 4)
+    assert (d.tokens.cpu().numpy() == od["tokens"]).all()

@@ -251,6 +251,20 @@ def run_native(args):
             for j in range(3):
                 stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
         stage_ms = [x / steps for x in stage_ms]
+    # timed region 4 (not part of the step): the draft-token draws that precede a verification call
+    draft_ms = None
+    if not args.no_call_events:
+        dws = torch.empty(max(fef.fef_draft_sample_workspace_bytes(w.B, w.K, w.V, w.dtype), 256), dtype=torch.uint8,
+                          device=dev)
+        dout = fef.fef_draft_sample(sets[0][0], w.temperature, seed, 0, workspace=dws)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        d0.record(stream)
+        for i in range(steps):
+            fef.fef_draft_sample(sets[i % nbuf][0], w.temperature, seed, i, out=dout, workspace=dws)
+        d1.record(stream)
+        barrier()
+        draft_ms = d0.elapsed_time(d1) / steps
     sampler.stop()
     status = int(out.device_status.item())
     accept_mean = float(out.accept_len.float().mean().item())
@@ -354,6 +368,11 @@ def run_native(args):
         "e2e": {"value": positions_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "api": "fef_spec_verify_host + fef_remask_select_host (pinned host buffers)"},
+        "draft_sample": None if draft_ms is None else {
+            "ms_per_call": draft_ms, "positions_per_s": w.B * w.K / (draft_ms * 1e-3),
+            "gbs": w.B * w.K * w.V * w.logit_bytes / (draft_ms * 1e-3) / 1e9,
+            "note": "fef_draft_sample on the draft logits of the same workload; bound by Philox arithmetic, not "
+                    "by HBM; not part of the step"},
         "gpu_launches": steps * 4,
         "clocks": sampler.result(),
         "cpu_baseline": cpu_baseline,

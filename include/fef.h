@@ -115,6 +115,27 @@ fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
                            int32_t* device_status, void* cuda_stream);
 
 /*
+ * fef_spec_verify for drafts that come with their law's normaliser (same operation, same
+ * citations: Algorithm 2's verification loop, Section 3.2).  `draft_log2_norm` is the
+ * log2_norm output of fef_draft_sample for the same draft_logits and temperature:
+ * rho_i(x) = 2^(l_x * log2(e) / T - draft_log2_norm[b,i]).  With it the draft rows need not be
+ * read in full: only draft_logits[b,i,x_i] is, and the rejected position's row for the residual
+ * draw, so a call moves half the bytes.  Results equal fef_spec_verify's up to the rounding of the
+ * normaliser (confidences within 1e-5 relative, the same draws apart from near-ties).
+ *   draft_log2_norm  device, [B, K] float64 (entries of positions i >= n_b are not read);
+ *                    a NaN or infinite entry is FEF_ERR_NONFINITE for its window
+ * Everything else as in fef_spec_verify; at temperature 0 the normalisers are not used.
+ */
+fef_status fef_spec_verify_with_draft_norm(const void* draft_logits, const void* target_logits,
+                                           const int32_t* draft_tokens, const double* draft_log2_norm,
+                                           const int32_t* row_len,
+                                           int B, int K, int V, int64_t ld, fef_dtype dt,
+                                           float temperature, uint64_t seed, uint32_t step,
+                                           int32_t* accept_len, int32_t* tokens, float* conf,
+                                           void* workspace, size_t workspace_bytes,
+                                           int32_t* device_status, void* cuda_stream);
+
+/*
  * fef_spec_verify with timing marks: the same operation (Algorithm 2's verification
  * loop) and the same results, and additionally up to four caller-created CUDA events
  * (cudaEvent_t passed as void*; NULL entries are skipped) are recorded on `cuda_stream`:

@@ -25,7 +25,7 @@ FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
 EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_spec_verify_profiled",
            "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static",
-           "fef_draft_sample_workspace_bytes", "fef_draft_sample")
+           "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm")
 
 _lib = None
 
@@ -57,6 +57,9 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_workspace_bytes.restype = sz
     L.fef_spec_verify.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, sz, vp, vp]
     L.fef_spec_verify.restype = i32
+    L.fef_spec_verify_with_draft_norm.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp,
+                                                  vp, sz, vp, vp]
+    L.fef_spec_verify_with_draft_norm.restype = i32
     L.fef_spec_verify_profiled.argtypes = L.fef_spec_verify.argtypes + [vp]
     L.fef_spec_verify_profiled.restype = i32
     L.fef_spec_verify_host_arena_bytes.argtypes = [i32, i32, i32, i64, i32]
@@ -119,12 +122,15 @@ class VerifyResult(NamedTuple):
 def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, draft_tokens: torch.Tensor,
                     temperature: float, seed: int, step: int, row_len: Optional[torch.Tensor] = None,
                     V: Optional[int] = None, out: Optional[VerifyResult] = None,
-                    workspace: Optional[torch.Tensor] = None, stream=None, stage_events=None) -> VerifyResult:
+                    workspace: Optional[torch.Tensor] = None, stream=None, stage_events=None,
+                    draft_log2_norm: Optional[torch.Tensor] = None) -> VerifyResult:
     """Enqueue one verification call (see ``fef_spec_verify`` in include/fef.h).
 
     With ``stage_events`` (four ``torch.cuda.Event(enable_timing=True)`` that have
     been recorded once, or ``None`` entries) the call goes through
-    ``fef_spec_verify_profiled`` and the events mark the kernel boundaries.
+    ``fef_spec_verify_profiled`` and the events mark the kernel boundaries.  With
+    ``draft_log2_norm`` (the ``log2_norm`` of ``fef_draft_sample``, ``[B, K]`` float64) the
+    call goes through ``fef_spec_verify_with_draft_norm`` and streams the target rows only.
 
     ``draft_logits`` / ``target_logits``: ``[B, K, ld]`` CUDA tensors, float32 or
     bfloat16, contiguous; ``V`` (default ``ld``) entries of each row are used.
@@ -156,7 +162,12 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
                 int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
                 out.accept_len.data_ptr(), out.tokens.data_ptr(), out.conf.data_ptr(),
                 workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(), _stream_ptr(stream))
-        if stage_events is None:
+        if draft_log2_norm is not None:
+            if draft_log2_norm.dtype != torch.float64 or draft_log2_norm.numel() != B * K or \
+                    not draft_log2_norm.is_contiguous() or draft_log2_norm.device != dev:
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm")
+            st = load().fef_spec_verify_with_draft_norm(*args[:3], draft_log2_norm.data_ptr(), *args[3:])
+        elif stage_events is None:
             st = load().fef_spec_verify(*args)
         else:
             handles = (ctypes.c_void_p * 4)(*[None if e is None else e.cuda_event for e in stage_events])

@@ -26,7 +26,8 @@ namespace fef {
 // Work split of one call, computed on the host and passed by value to the kernels.
 struct Geometry {
     int B, K, V;
-    int units_per_row;    // 2: target row and draft row; 1 in greedy mode (target only)
+    int units_per_row;    // 2: target row and draft row; 1 when only the target rows are streamed (greedy
+                          // mode, or the draft laws' normalisers are given)
     int tile_bytes;       // bytes of one streaming tile (8, 16 or 32 KiB)
     int vec_bytes;        // bytes of a row covered by whole 16-byte vectors
     int vec_elems;        // the same in elements; elements beyond are the row's "tail"
@@ -46,6 +47,7 @@ struct VerifyParams {
     const char* draft;    // q logits
     const int32_t* draft_tokens;
     const int32_t* row_len;
+    const double* draft_norm;  // [B*K] log2 normalisers of the draft laws, or null: stream the draft rows
     float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
@@ -505,10 +507,18 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
             const char* prow = P.target + row * G.ld_bytes;
             const char* qrow = P.draft + row * G.ld_bytes;
             const int x = tok[r];
-            const RowNorm np = fold_unit<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P);
+            const RowNorm np = fold_unit<DT, GREEDY>(row * G.units_per_row, prow, c, P);
             RowNorm nq;
             nq.bad = false;
-            if constexpr (!GREEDY) nq = fold_unit<DT, false>(2 * row + 1, qrow, c, P);
+            if constexpr (!GREEDY) {
+                if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
+                    nq.M = P.draft_norm[row];
+                    nq.S = 1.0;
+                    nq.bad = !(fabs(nq.M) < INFINITY);
+                } else {
+                    nq = fold_unit<DT, false>(2 * row + 1, qrow, c, P);
+                }
+            }
             if (x < 0 || x >= G.V) {
                 err = max(err, static_cast<int>(FEF_ERR_TOKEN_RANGE));
             } else if (np.bad || nq.bad) {
@@ -693,10 +703,18 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
         const int64_t row = static_cast<int64_t>(b) * G.K + i;
         const char* prow = P.target + row * G.ld_bytes;
         const char* qrow = P.draft + row * G.ld_bytes;
-        const RowNorm np = fold_unit_warp<DT, GREEDY>(GREEDY ? row : 2 * row, prow, c, P, lane);
+        const RowNorm np = fold_unit_warp<DT, GREEDY>(row * G.units_per_row, prow, c, P, lane);
         RowNorm nq;
         nq.bad = false;
-        if constexpr (!GREEDY) nq = fold_unit_warp<DT, false>(2 * row + 1, qrow, c, P, lane);
+        if constexpr (!GREEDY) {
+            if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
+                nq.M = P.draft_norm[row];
+                nq.S = 1.0;
+                nq.bad = !(fabs(nq.M) < INFINITY);
+            } else {
+                nq = fold_unit_warp<DT, false>(2 * row + 1, qrow, c, P, lane);
+            }
+        }
         if (lane == 0) {
             const int x = __ldg(P.draft_tokens + row);
             int err = 0, accept = 0, alt = -1;
@@ -1022,7 +1040,8 @@ static int sm_count_of_current_device(int* device_out) {
     return g_sm_count[dev];
 }
 
-static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool greedy, int sm_count, Geometry* out) {
+static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool target_only, int sm_count,
+                          Geometry* out) {
     if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V || sm_count < 1) return false;
     if (dt != FEF_F32 && dt != FEF_BF16) return false;
     const int esize = dt == FEF_F32 ? 4 : 2;
@@ -1031,7 +1050,7 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool gr
     G.B = B;
     G.K = K;
     G.V = V;
-    G.units_per_row = greedy ? 1 : 2;
+    G.units_per_row = target_only ? 1 : 2;
     G.ld_bytes = ld * esize;
     G.vec_bytes = static_cast<int>((static_cast<int64_t>(V) * esize) / 16 * 16);
     G.vec_elems = G.vec_bytes / esize;
@@ -1179,12 +1198,14 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
     return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
 }
 
-fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
-                                    const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
-                                    int64_t ld, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
-                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
-                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
-                                    void* const* stage_events) {
+}  // extern "C"
+
+// Every verification entry point ends here.
+static fef_status verify_impl(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                              const int32_t* row_len, const double* draft_log2_norm, int B, int K, int V, int64_t ld,
+                              fef_dtype dt, float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                              int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                              int32_t* device_status, void* cuda_stream, void* const* stage_events) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -1203,7 +1224,7 @@ fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target
     const bool greedy = (temperature == 0.0f);
 
     VerifyParams P;
-    if (!make_geometry(B, K, V, ld, dt, greedy, sms, &P.geo)) return FEF_ERR_INVALID_ARG;
+    if (!make_geometry(B, K, V, ld, dt, greedy || draft_log2_norm != nullptr, sms, &P.geo)) return FEF_ERR_INVALID_ARG;
     const WorkspaceLayout L = layout_of(P.geo);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return FEF_ERR_WORKSPACE;
@@ -1227,6 +1248,7 @@ fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target
     P.draft = static_cast<const char*>(draft_logits);
     P.draft_tokens = draft_tokens;
     P.row_len = row_len;
+    P.draft_norm = greedy ? nullptr : draft_log2_norm;
     P.seed = seed;
     P.step = step;
     P.accept_len = accept_len;
@@ -1254,14 +1276,38 @@ fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target
     return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
+extern "C" {
+
+fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const int32_t* row_len, int B, int K, int V,
+                                    int64_t ld, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
+                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
+                                    void* const* stage_events) {
+    return verify_impl(draft_logits, target_logits, draft_tokens, row_len, nullptr, B, K, V, ld, dt, temperature, seed,
+                       step, accept_len, tokens, conf, workspace, workspace_bytes, device_status, cuda_stream,
+                       stage_events);
+}
+
 fef_status fef_spec_verify(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
                            const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
                            float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
                            int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
                            int32_t* device_status, void* cuda_stream) {
-    return fef_spec_verify_profiled(draft_logits, target_logits, draft_tokens, row_len, B, K, V, ld, dt,
-                                    temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes,
-                                    device_status, cuda_stream, nullptr);
+    return verify_impl(draft_logits, target_logits, draft_tokens, row_len, nullptr, B, K, V, ld, dt, temperature, seed,
+                       step, accept_len, tokens, conf, workspace, workspace_bytes, device_status, cuda_stream, nullptr);
+}
+
+fef_status fef_spec_verify_with_draft_norm(const void* draft_logits, const void* target_logits,
+                                           const int32_t* draft_tokens, const double* draft_log2_norm,
+                                           const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                                           float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
+                                           int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
+                                           int32_t* device_status, void* cuda_stream) {
+    if (!draft_log2_norm) return FEF_ERR_INVALID_ARG;
+    return verify_impl(draft_logits, target_logits, draft_tokens, row_len, draft_log2_norm, B, K, V, ld, dt,
+                       temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes, device_status,
+                       cuda_stream, nullptr);
 }
 
 // ---- host-buffer variant: layout of the caller's device arena

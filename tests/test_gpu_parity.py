@@ -437,3 +437,27 @@ def test_draft_tokens_feed_verification(fef):
     _check(fef, q, p, d.tokens, 0.7, 31, 4)
     od = oracle.draft_sample(q.cpu(), 0.7, 31, 4)
     assert (d.tokens.cpu().numpy() == od["tokens"]).all()
+
+
+def test_verification_with_the_draft_normalisers_streams_the_target_only(fef):
+    """fef_draft_sample -> fef_spec_verify_with_draft_norm against the oracle pair, and against the plain call."""
+    for w, T, seed in ((synth.LLADA_BATCHED.with_(B=5, K=16), 0.7, 41), (synth.LLADA_SINGLE.with_(K=8), 1.0, 42),
+                       (synth.DREAM_LARGE.with_(B=3, K=8, dtype=torch.float32), 1.0, 43)):
+        q, p = synth.make_logits(w, seed=seed, device="cuda")
+        d = fef.fef_draft_sample(q, T, seed, 7)
+        r = fef.fef_spec_verify(q, p, d.tokens, T, seed, 7, draft_log2_norm=d.log2_norm)
+        plain = fef.fef_spec_verify(q, p, d.tokens, T, seed, 7)
+        torch.cuda.synchronize()
+        assert int(r.device_status.item()) == 0
+        ref = oracle.spec_verify(q.cpu(), p.cpu(), d.tokens.cpu(), T, seed, 7)
+        rep = compare_verify(r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy(), ref)
+        assert rep.ok, rep.mismatches[:5]
+        assert (r.accept_len == plain.accept_len).all() and (r.tokens == plain.tokens).all()
+        assert torch.allclose(r.conf, plain.conf, rtol=1e-5, atol=0)
+    # a bad normaliser poisons its window only
+    bad = d.log2_norm.clone()
+    bad[1, 0] = float("nan")
+    r = fef.fef_spec_verify(q, p, d.tokens, T, seed, 7, draft_log2_norm=bad)
+    torch.cuda.synchronize()
+    assert int(r.device_status.item()) == fef.FEF_ERR_NONFINITE
+    assert r.accept_len[1].item() == -1 and (r.accept_len[[0, 2]] == plain.accept_len[[0, 2]]).all()

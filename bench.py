@@ -252,7 +252,7 @@ def run_native(args):
                 stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
         stage_ms = [x / steps for x in stage_ms]
     # timed region 4 (not part of the step): the draft-token draws that precede a verification call
-    draft_ms = None
+    draft_ms = norm_ms = None
     if not args.no_call_events:
         dws = torch.empty(max(fef.fef_draft_sample_workspace_bytes(w.B, w.K, w.V, w.dtype), 256), dtype=torch.uint8,
                           device=dev)
@@ -265,6 +265,17 @@ def run_native(args):
         d1.record(stream)
         barrier()
         draft_ms = d0.elapsed_time(d1) / steps
+        # ... and the verification that reuses their normalisers (streams the target rows only)
+        douts = [fef.fef_draft_sample(sets[i][0], w.temperature, seed, 0) for i in range(nbuf)]
+        barrier()
+        d0.record(stream)
+        for i in range(steps):
+            q, p, _ = sets[i % nbuf]
+            fef.fef_spec_verify(q, p, douts[i % nbuf].tokens, w.temperature, seed, 0, out=out, workspace=ws,
+                                draft_log2_norm=douts[i % nbuf].log2_norm)
+        d1.record(stream)
+        barrier()
+        norm_ms = d0.elapsed_time(d1) / steps
     sampler.stop()
     status = int(out.device_status.item())
     accept_mean = float(out.accept_len.float().mean().item())
@@ -372,7 +383,9 @@ def run_native(args):
             "ms_per_call": draft_ms, "positions_per_s": w.B * w.K / (draft_ms * 1e-3),
             "gbs": w.B * w.K * w.V * w.logit_bytes / (draft_ms * 1e-3) / 1e9,
             "note": "fef_draft_sample on the draft logits of the same workload; bound by Philox arithmetic, not "
-                    "by HBM; not part of the step"},
+                    "by HBM; not part of the step",
+            "verify_with_draft_norm_ms": norm_ms,
+            "verify_with_draft_norm_positions_per_s": w.B * w.K / (norm_ms * 1e-3)},
         "gpu_launches": steps * 4,
         "clocks": sampler.result(),
         "cpu_baseline": cpu_baseline,

@@ -461,3 +461,54 @@ def test_verification_with_the_draft_normalisers_streams_the_target_only(fef):
     torch.cuda.synchronize()
     assert int(r.device_status.item()) == fef.FEF_ERR_NONFINITE
     assert r.accept_len[1].item() == -1 and (r.accept_len[[0, 2]] == plain.accept_len[[0, 2]]).all()
+
+
+# ------------------------------------------------- long-generation sweep ----
+@pytest.mark.parametrize("B,K,dtype", [(1, 8, torch.float32), (8, 64, torch.bfloat16), (8, 8, torch.bfloat16),
+                                       (1, 64, torch.float32), (8, 32, torch.float32)])
+def test_long_generation_sweep_points(fef, B, K, dtype):
+    """Config 4 (gen length 1024, V = 126464, logits regenerated on the device every round, full
+    loop of draft draws, verification and re-masking until nothing is masked), two denoising
+    steps.  Drafts come from fef_draft_sample, verification reuses their normalisers on odd
+    rounds and streams both tensors on even rounds.  The oracle re-verifies the device's
+    inputs on a fixed sample of rounds (the first three, then every 40th; all windows)."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop
+
+    w = synth.HEADLINE.with_(B=B, K=K, dtype=dtype, noise_std=0.7)
+    L = 1024
+    total = ParityReport()
+    state = {}
+
+    def logits_fn(rnd, window, row_len):
+        return synth.make_logits(w, seed=7000 + rnd, device="cuda")
+
+    def draft_fn(q, rnd):
+        state["draft"] = fef.fef_draft_sample(q, w.temperature, 77, rnd)
+        return state["draft"].tokens
+
+    def verify_fn(q, p, tok, rl, rnd):
+        norm = state["draft"].log2_norm if rnd % 2 else None
+        r = fef.fef_spec_verify(q, p, tok, w.temperature, 77, rnd, row_len=rl, draft_log2_norm=norm)
+        torch.cuda.synchronize()
+        assert int(r.device_status.item()) == 0
+        ga, gt, gc = r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy()
+        if rnd < 3 or rnd % 40 == 0:
+            od = oracle.draft_sample(q.cpu(), w.temperature, 77, rnd)
+            used = np.arange(K)[None, :] < rl.cpu().numpy()[:, None]
+            assert (tok.cpu().numpy()[used] == od["tokens"][used]).all()
+            ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), w.temperature, 77, rnd, row_len=rl.cpu())
+            rep = compare_verify(ga, gt, gc, ref)
+            assert rep.ok, rep.mismatches[:5]
+            total.merge(rep)
+        return ga, gt, gc
+
+    def select_fn(conf, mask, k):
+        pos, cnt = fef.fef_remask_select(conf, mask, k)
+        opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
+        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
+        return opos, ocnt
+
+    out = run_decode_loop(B, L, K, 2, 8, logits_fn, draft_fn, verify_fn, select_fn)
+    assert (out["tokens"] >= 0).all()
+    assert total.windows >= 3 * B
+    print(total.summary(), "rounds", out["rounds"])

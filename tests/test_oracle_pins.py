@@ -612,3 +612,72 @@ def test_draft_sample_zero_probability_entries_row_len_and_errors():
     assert out["tokens"][0, 0] == -1 and out["tokens"][1, 0] == -1 and out["tokens"][2, 0] >= 0
     bf = torch.tensor(np.random.default_rng(1).normal(0, 2, size=(4, 2, 33)).astype(np.float32)).to(torch.bfloat16)
     assert (oracle.draft_sample(bf, 0.9, 5, 5)["tokens"] == oracle.draft_sample(bf.float(), 0.9, 5, 5)["tokens"]).all()
+
+
+# ------------------------------------------------- Algorithm 2 bookkeeping ----
+from oracle import loop as oloop  # noqa: E402
+
+
+def test_loop_window_is_the_first_unresolved_positions_in_order():
+    rng = np.random.default_rng(0)
+    for B, L, K in ((1, 1, 1), (3, 17, 4), (2, 64, 64), (4, 100, 8)):
+        tokens = np.where(rng.random((B, L)) < 0.4, oloop.MASK, rng.integers(0, 50, (B, L))).astype(np.int32)
+        tokens[0, :] = 7 if B > 1 else tokens[0]          # a fully resolved row
+        win, rl, unres = oloop.next_window(tokens, K)
+        for b in range(B):
+            masked = np.nonzero(tokens[b] == oloop.MASK)[0]
+            assert unres[b] == len(masked) and rl[b] == min(K, len(masked))
+            assert (win[b, :rl[b]] == masked[:K]).all() and (win[b, rl[b]:] == -1).all()
+
+
+def test_loop_verification_inputs_use_verified_prefix_and_draft_prefix():
+    tokens = np.array([[5, -1, 6, -1, -1, 9]], dtype=np.int32)
+    win, rl, _ = oloop.next_window(tokens, 3)
+    drafts = np.array([[11, 12, 13]], dtype=np.int32)
+    X = oloop.verification_inputs(tokens, win, rl, drafts)
+    assert X[0, 0].tolist() == [5, -1, 6, -1, -1, 9]          # m = 0: nothing drafted yet
+    assert X[0, 1].tolist() == [5, 11, 6, -1, -1, 9]          # m = 1: x~_{j_0} in place
+    assert X[0, 2].tolist() == [5, 11, 6, 12, -1, 9]          # m = 2: x~_{j_0}, x~_{j_1}; j_2 itself still masked
+    # the input of position j_m never holds its own draft or later ones
+    for m in range(3):
+        assert X[0, m, win[0, m]] == oloop.MASK
+
+
+def test_loop_commit_counts_match_theorem_2_and_remask_restores_masks():
+    tokens = np.full((3, 8), oloop.MASK, dtype=np.int32)
+    conf = np.full((3, 8), -1.0, dtype=np.float32)
+    in_step = np.zeros((3, 8), dtype=np.uint8)
+    win, rl, _ = oloop.next_window(tokens, 4)
+    accept = np.array([2, 4, -1], dtype=np.int32)              # reject at 2; all 4 accepted; data error
+    out_tok = np.arange(12, dtype=np.int32).reshape(3, 4) + 100
+    out_conf = np.linspace(0.1, 0.9, 12, dtype=np.float32).reshape(3, 4)
+    committed = oloop.commit(tokens, conf, in_step, win, rl, accept, out_tok, out_conf)
+    assert committed.tolist() == [3, 4, -1]                    # a + 1 with the corrected token; n when none rejected
+    assert tokens[0].tolist() == [100, 101, 102, -1, -1, -1, -1, -1] and tokens[2].tolist() == [-1] * 8
+    assert in_step.sum(axis=1).tolist() == [3, 4, 0]
+    pos = np.array([[1, 0], [3, -1], [-1, -1]], dtype=np.int32)
+    oloop.remask(tokens, conf, in_step, pos, np.array([2, 1, 0], dtype=np.int32))
+    assert tokens[0, :3].tolist() == [-1, -1, 102] and tokens[1, 3] == -1 and conf[0, 0] == -1.0
+    assert in_step.sum() == 0
+
+
+def test_loop_toy_run_resolves_everything_and_remasks_the_lowest_confidences():
+    rng = np.random.default_rng(3)
+    B, L, K, k = 2, 20, 4, 3
+    tokens = np.full((B, L), oloop.MASK, dtype=np.int32)
+    conf = np.full((B, L), -1.0, dtype=np.float32)
+    in_step = np.zeros((B, L), dtype=np.uint8)
+    rounds = 0
+    while (tokens == oloop.MASK).any():
+        win, rl, _ = oloop.next_window(tokens, K)
+        a = np.minimum(rng.integers(0, K + 1, B), rl).astype(np.int32)
+        committed = oloop.commit(tokens, conf, in_step, win, rl, a, rng.integers(0, 99, (B, K)).astype(np.int32),
+                                 rng.random((B, K)).astype(np.float32))
+        assert (committed == np.minimum(a + 1, rl)).all()
+        rounds += 1
+        assert rounds < 100
+    pos, cnt = oracle.remask_select(conf, in_step, k)
+    for b in range(B):
+        assert sorted(pos[b].tolist()) == sorted(np.argsort(conf[b], kind="stable")[:k].tolist())
+    oloop.remask(tokens, conf, in_step, pos, cnt)
+    assert ((tokens == oloop.MASK).sum(axis=1) == k).all()

@@ -49,6 +49,8 @@ typedef enum { FEF_F32 = 0, FEF_BF16 = 1 } fef_dtype;
 #define FEF_MAX_B 65535
 #define FEF_MAX_K 64
 #define FEF_MAX_REMASK_L 8192
+/* Token id of a masked (unresolved) position in the decode-loop state. */
+#define FEF_MASK_TOKEN (-1)
 
 /* Human-readable name of a status value (static storage, never NULL). */
 const char* fef_status_string(fef_status s);
@@ -267,6 +269,38 @@ size_t fef_remask_select_host_arena_bytes(int B, int L, int k);
 fef_status fef_remask_select_host(const float* conf, const uint8_t* mask, int B, int L, int k,
                                   int32_t* positions, int32_t* count,
                                   void* device_arena, size_t device_arena_bytes, void* cuda_stream);
+
+/*
+ * Bookkeeping of the full-sequence decoding loop (Algorithm 2) on the device.  State of B
+ * sequences of L positions: tokens [B, L] int32 (FEF_MASK_TOKEN = unresolved), conf [B, L]
+ * float32 (-1 where unresolved), in_step [B, L] uint8 (1 = committed during the current
+ * denoising step, the set C^(s)).  All pointers are device memory; every call is one small
+ * kernel on `cuda_stream`.  1 <= L <= 2^24, 1 <= K <= FEF_MAX_K.
+ *
+ * fef_loop_next_window  ("Let J_t be the unresolved positions, j_1 < ... < j_Lt; b = min{k, L_t}"):
+ *   window_pos [B, K] = the first K unresolved positions of each row in increasing order, -1
+ *   padded; row_len [B] = min(K, L_t); unresolved [B] = L_t.
+ * fef_loop_verification_inputs  ("Construct verification inputs X^(j_m) ... each input uses the
+ *   verified prefix and the draft prefix x~_{j_1} .. x~_{j_{m-1}}"): inputs [B, K, L]; row m is
+ *   the sequence with the drafts of the window's positions 0 .. min(m, row_len) - 1 written in.
+ * fef_loop_commit  ("X^{j_m} <- x~ or Z; C^(s) <- C^(s) u {(j_m, c_{j_m})}; discard the remaining
+ *   drafts"): writes the first min(accept_len + 1, row_len) entries of out_tokens / out_conf
+ *   (outputs of fef_spec_verify) to their positions, marks them in in_step; committed [B] = that
+ *   count, or -1 (nothing written) for a window with accept_len = -1.
+ * fef_loop_remask  ("Re-corrupt X^i for i in LowConf(C^(s))", absorbing-state kernel): the first
+ *   min(count[b], k) entries of positions [B, k] (output of fef_remask_select) go back to
+ *   FEF_MASK_TOKEN with conf -1; in_step is cleared for the next denoising step.
+ */
+fef_status fef_loop_next_window(const int32_t* tokens, int B, int L, int K,
+                                int32_t* window_pos, int32_t* row_len, int32_t* unresolved, void* cuda_stream);
+fef_status fef_loop_verification_inputs(const int32_t* tokens, const int32_t* window_pos, const int32_t* row_len,
+                                        const int32_t* draft_tokens, int B, int L, int K,
+                                        int32_t* inputs, void* cuda_stream);
+fef_status fef_loop_commit(const int32_t* window_pos, const int32_t* row_len, const int32_t* accept_len,
+                           const int32_t* out_tokens, const float* out_conf, int B, int L, int K,
+                           int32_t* tokens, float* conf, uint8_t* in_step, int32_t* committed, void* cuda_stream);
+fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B, int L, int k,
+                           int32_t* tokens, float* conf, uint8_t* in_step, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ FEF_MAX_K, FEF_MAX_REMASK_L = 64, 8192
 EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_verify", "fef_spec_verify_profiled",
            "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static",
-           "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm")
+           "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm",
+           "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask")
 
 _lib = None
 
@@ -72,6 +73,12 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_draft_sample_workspace_bytes.restype = sz
     L.fef_draft_sample.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.fef_draft_sample.restype = i32
+    L.fef_loop_next_window.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+    L.fef_loop_verification_inputs.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp]
+    L.fef_loop_commit.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.fef_loop_remask.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    for fn in (L.fef_loop_next_window, L.fef_loop_verification_inputs, L.fef_loop_commit, L.fef_loop_remask):
+        fn.restype = i32
     L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.fef_remask_select.restype = i32
     L.fef_remask_select_host_arena_bytes.argtypes = [i32, i32, i32]
@@ -165,7 +172,8 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
         if draft_log2_norm is not None:
             if draft_log2_norm.dtype != torch.float64 or draft_log2_norm.numel() != B * K or \
                     not draft_log2_norm.is_contiguous() or draft_log2_norm.device != dev:
-                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm")
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm",
+           "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask")
             st = load().fef_spec_verify_with_draft_norm(*args[:3], draft_log2_norm.data_ptr(), *args[3:])
         elif stage_events is None:
             st = load().fef_spec_verify(*args)
@@ -222,6 +230,73 @@ def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, 
     if st != FEF_OK:
         raise FefError(st, "fef_draft_sample")
     return out
+
+
+MASK_TOKEN = -1
+
+
+def _i32_cuda(t: torch.Tensor, where: str):
+    if t.device.type != "cuda" or t.dtype != torch.int32 or not t.is_contiguous():
+        raise FefError(FEF_ERR_INVALID_ARG, where)
+    return t
+
+
+def fef_loop_next_window(tokens: torch.Tensor, K: int, stream=None):
+    """``tokens [B, L]`` int32 -> ``(window_pos [B, K], row_len [B], unresolved [B])`` (see include/fef.h)."""
+    _i32_cuda(tokens, "fef_loop_next_window")
+    B, L = tokens.shape
+    dev = tokens.device
+    with torch.cuda.device(dev):
+        window = torch.empty((B, K), dtype=torch.int32, device=dev)
+        row_len = torch.empty(B, dtype=torch.int32, device=dev)
+        unresolved = torch.empty(B, dtype=torch.int32, device=dev)
+        st = load().fef_loop_next_window(tokens.data_ptr(), B, L, K, window.data_ptr(), row_len.data_ptr(),
+                                         unresolved.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_next_window")
+    return window, row_len, unresolved
+
+
+def fef_loop_verification_inputs(tokens, window_pos, row_len, draft_tokens, stream=None) -> torch.Tensor:
+    """The K verification inputs X^(j_m) of every window, ``[B, K, L]`` int32 (see include/fef.h)."""
+    for t in (tokens, window_pos, row_len, draft_tokens):
+        _i32_cuda(t, "fef_loop_verification_inputs")
+    B, L = tokens.shape
+    K = window_pos.shape[1]
+    with torch.cuda.device(tokens.device):
+        out = torch.empty((B, K, L), dtype=torch.int32, device=tokens.device)
+        st = load().fef_loop_verification_inputs(tokens.data_ptr(), window_pos.data_ptr(), row_len.data_ptr(),
+                                                 draft_tokens.data_ptr(), B, L, K, out.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_verification_inputs")
+    return out
+
+
+def fef_loop_commit(window_pos, row_len, verified: "VerifyResult", tokens, conf, in_step, stream=None) -> torch.Tensor:
+    """Write one verification result back into the loop state (in place); returns ``committed [B]``."""
+    for t in (window_pos, row_len, tokens):
+        _i32_cuda(t, "fef_loop_commit")
+    B, L = tokens.shape
+    K = window_pos.shape[1]
+    with torch.cuda.device(tokens.device):
+        committed = torch.empty(B, dtype=torch.int32, device=tokens.device)
+        st = load().fef_loop_commit(window_pos.data_ptr(), row_len.data_ptr(), verified.accept_len.data_ptr(),
+                                    verified.tokens.data_ptr(), verified.conf.data_ptr(), B, L, K, tokens.data_ptr(),
+                                    conf.data_ptr(), in_step.data_ptr(), committed.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_commit")
+    return committed
+
+
+def fef_loop_remask(positions, count, tokens, conf, in_step, stream=None) -> None:
+    """Send the selected positions back to MASK and empty the step's set (in place)."""
+    B, L = tokens.shape
+    k = positions.shape[1]
+    with torch.cuda.device(tokens.device):
+        st = load().fef_loop_remask(positions.data_ptr() if k else None, count.data_ptr(), B, L, k, tokens.data_ptr(),
+                                    conf.data_ptr(), in_step.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_remask")
 
 
 def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions: Optional[torch.Tensor] = None,
@@ -359,6 +434,7 @@ def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena
     return positions, count
 
 
-__all__ = ["fef_draft_sample", "fef_draft_sample_workspace_bytes", "DraftResult", "fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
+__all__ = ["fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask", "MASK_TOKEN",
+           "fef_draft_sample", "fef_draft_sample_workspace_bytes", "DraftResult", "fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libfef.so")
-SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu"]
+SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu", "fef_loop.cu"]
 HEADERS = [os.path.join(CSRC, "fef_common.cuh"), os.path.join(CSRC, "fef_device_math.cuh"), os.path.join(INCLUDE, "fef.h")]
 
 

@@ -80,3 +80,59 @@ def run_decode_loop(B: int, L: int, K: int, n_steps: int, remask_k: int,
                 tokens[b, sel] = MASK
                 conf[b, sel] = -1.0
     return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist)
+
+
+def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: int, logits_fn: Callable,
+                           temperature: float, seed: int, on_round: Optional[Callable] = None,
+                           first_round: int = 0, reuse_draft_norm: bool = True, build_inputs: bool = False):
+    """Algorithm 2 with the whole state resident on the device: every step of a round is one
+    library call (``fef_loop_next_window`` -> [``fef_loop_verification_inputs``] ->
+    ``fef_draft_sample`` -> ``fef_spec_verify`` -> ``fef_loop_commit``), and a denoising step ends
+    with ``fef_remask_select`` + ``fef_loop_remask``.  The host reads back one integer per round
+    (the largest count of unresolved positions) to know when the step is over.
+
+    ``fef`` is the binding module.  logits_fn(round, window_pos [B,K] int32 CUDA, row_len [B] int32
+    CUDA, inputs [B,K,L] int32 CUDA or None) -> (draft_logits, target_logits), both [B,K,V] CUDA.
+    on_round(round, dict of the round's device tensors): optional hook, called after the commit with
+    the state before it under "before"; called with round None after each re-masking.
+
+    Returns dict(tokens [B,L] int32, conf [B,L] float32 (CUDA), rounds, committed_per_round).
+    """
+    dev = torch.device("cuda")
+    tokens = torch.full((B, L), MASK, dtype=torch.int32, device=dev)
+    conf = torch.full((B, L), -1.0, dtype=torch.float32, device=dev)
+    in_step = torch.zeros((B, L), dtype=torch.uint8, device=dev)
+    rnd = first_round
+    committed_hist = []
+    for s in range(n_steps):
+        while True:
+            window, row_len, unresolved = fef.fef_loop_next_window(tokens, K)
+            if int(unresolved.max().item()) == 0:
+                break
+            inputs = None
+            q, p = logits_fn(rnd, window, row_len, None)
+            draft = fef.fef_draft_sample(q, temperature, seed, rnd, row_len=row_len)
+            if build_inputs:
+                inputs = fef.fef_loop_verification_inputs(tokens, window, row_len, draft.tokens)
+            norm = draft.log2_norm if reuse_draft_norm else None
+            res = fef.fef_spec_verify(q, p, draft.tokens, temperature, seed, rnd, row_len=row_len,
+                                      draft_log2_norm=norm)
+            before = (tokens.clone(), conf.clone(), in_step.clone()) if on_round is not None else None
+            committed = fef.fef_loop_commit(window, row_len, res, tokens, conf, in_step)
+            if on_round is not None:
+                on_round(rnd, dict(q=q, p=p, draft=draft, window=window, row_len=row_len, unresolved=unresolved,
+                                   inputs=inputs, result=res, committed=committed, before=before,
+                                   tokens=tokens, conf=conf, in_step=in_step))
+            n = committed.cpu()
+            if (n < 0).any():
+                raise RuntimeError("verification reported a data error in round %d" % rnd)
+            committed_hist.append(int(n.sum()))
+            rnd += 1
+        if s < n_steps - 1 and remask_k > 0:
+            positions, count = fef.fef_remask_select(conf, in_step, remask_k)
+            before = (tokens.clone(), conf.clone(), in_step.clone()) if on_round is not None else None
+            fef.fef_loop_remask(positions, count, tokens, conf, in_step)
+            if on_round is not None:
+                on_round(None, dict(positions=positions, count=count, before=before,
+                                    tokens=tokens, conf=conf, in_step=in_step))
+    return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist)

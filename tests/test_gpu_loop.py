@@ -1,0 +1,146 @@
+"""Device-resident bookkeeping of the decoding loop (Algorithm 2) against the CPU oracle (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import loop as oloop
+from oracle.compare import compare_verify
+from paper_2605_14305_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fef():
+    import paper_2605_14305_b200 as lib
+
+    lib.load(build_if_missing=True)
+    return lib
+
+
+def _random_state(B, L, frac_masked, seed):
+    rng = np.random.default_rng(seed)
+    tokens = rng.integers(0, 50000, size=(B, L)).astype(np.int32)
+    masked = rng.random((B, L)) < frac_masked
+    if B > 1:
+        masked[0] = False          # a finished row
+        masked[-1] = True          # a row that is still all masked
+    tokens[masked] = oloop.MASK
+    conf = rng.random((B, L)).astype(np.float32)
+    conf[masked] = -1.0
+    in_step = ((rng.random((B, L)) < 0.5) & ~masked).astype(np.uint8)
+    return tokens, conf, in_step
+
+
+@pytest.mark.parametrize("B,L,K", [(1, 1, 1), (2, 5, 4), (3, 256, 32), (4, 257, 7), (5, 1000, 64), (2, 4097, 64),
+                                   (64, 1024, 32), (1, 70000, 64)])
+@pytest.mark.parametrize("frac", [0.0, 0.03, 0.5, 1.0])
+def test_each_bookkeeping_call_matches_the_oracle(fef, B, L, K, frac):
+    tokens, conf, in_step = _random_state(B, L, frac, seed=B * 1000 + L + K)
+    rng = np.random.default_rng(L)
+    d_tokens, d_conf, d_in = (torch.as_tensor(x).cuda() for x in (tokens, conf, in_step))
+
+    # window
+    w, rl, un = fef.fef_loop_next_window(d_tokens, K)
+    ow, orl, oun = oloop.next_window(tokens, K)
+    assert (w.cpu().numpy() == ow).all() and (rl.cpu().numpy() == orl).all() and (un.cpu().numpy() == oun).all()
+
+    # verification inputs (kept small: B*K*L ints)
+    draft = rng.integers(0, 50000, size=(B, K)).astype(np.int32)
+    if B * K * L <= 1 << 24:
+        x = fef.fef_loop_verification_inputs(d_tokens, w, rl, torch.as_tensor(draft).cuda())
+        assert (x.cpu().numpy() == oloop.verification_inputs(tokens, ow, orl, draft)).all()
+
+    # commit: every accept length 0 .. K, and one failed window
+    accept = rng.integers(0, K + 1, size=B).astype(np.int32)
+    accept = np.minimum(accept, orl)               # what verification can return for this window
+    if B > 2:
+        accept[1] = -1
+    out_tok = rng.integers(0, 50000, size=(B, K)).astype(np.int32)
+    out_conf = rng.random((B, K)).astype(np.float32)
+    res = fef.VerifyResult(torch.as_tensor(accept).cuda(), torch.as_tensor(out_tok).cuda(),
+                           torch.as_tensor(out_conf).cuda(), torch.zeros(1, dtype=torch.int32, device="cuda"))
+    n = fef.fef_loop_commit(w, rl, res, d_tokens, d_conf, d_in)
+    on = oloop.commit(tokens, conf, in_step, ow, orl, accept, out_tok, out_conf)
+    assert (n.cpu().numpy() == on).all()
+    assert (d_tokens.cpu().numpy() == tokens).all() and (d_conf.cpu().numpy() == conf).all()
+    assert (d_in.cpu().numpy() == in_step).all()
+
+    # re-masking of LowConf's choice
+    for k in (0, 1, 8):
+        if k > L or L > fef.FEF_MAX_REMASK_L:
+            continue
+        pos, cnt = fef.fef_remask_select(d_conf, d_in, k)
+        opos, ocnt = oracle.remask_select(conf, in_step, k)
+        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
+        fef.fef_loop_remask(pos, cnt, d_tokens, d_conf, d_in)
+        oloop.remask(tokens, conf, in_step, opos, ocnt)
+        assert (d_tokens.cpu().numpy() == tokens).all() and (d_conf.cpu().numpy() == conf).all()
+        assert (d_in.cpu().numpy() == in_step).all()
+        in_step[:] = (tokens != oloop.MASK) & (rng.random((B, L)) < 0.5)
+        d_in.copy_(torch.as_tensor(in_step))
+
+
+def test_bookkeeping_argument_errors(fef):
+    t = torch.zeros((2, 8), dtype=torch.int32, device="cuda")
+    with pytest.raises(fef.FefError):
+        fef.fef_loop_next_window(t, 0)
+    with pytest.raises(fef.FefError):
+        fef.fef_loop_next_window(t, fef.FEF_MAX_K + 1)
+    with pytest.raises(fef.FefError):
+        fef.fef_loop_next_window(t.to(torch.int64), 4)
+    with pytest.raises(fef.FefError):
+        fef.fef_loop_next_window(t.cpu(), 4)
+
+
+@pytest.mark.parametrize("B,K,L,dtype,T", [(1, 4, 64, torch.float32, 1.0), (3, 8, 100, torch.bfloat16, 1.0),
+                                           (8, 32, 256, torch.bfloat16, 0.7), (2, 16, 96, torch.float32, 0.0)])
+def test_device_resident_loop_matches_the_oracle_round_by_round(fef, B, K, L, dtype, T):
+    """Three denoising steps with every call of every round re-done by the oracle on the device's
+    inputs: window, draft draws, verification, commit, LowConf and re-masking; the oracle keeps
+    its own copy of the state and the two must agree after every call."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device
+
+    w = synth.TINY.with_(B=B, K=K, V=2048, dtype=dtype, temperature=T, noise_std=0.6)
+    st = dict(tokens=np.full((B, L), oloop.MASK, dtype=np.int32), conf=np.full((B, L), -1.0, dtype=np.float32),
+              in_step=np.zeros((B, L), dtype=np.uint8), rounds=0, remasks=0)
+
+    def logits_fn(rnd, window, row_len, inputs):
+        return synth.make_logits(w, seed=300 + rnd, device="cuda")
+
+    def on_round(rnd, d):
+        if rnd is None:
+            opos, ocnt = oracle.remask_select(st["conf"], st["in_step"], 5)
+            assert (d["positions"].cpu().numpy() == opos).all() and (d["count"].cpu().numpy() == ocnt).all()
+            oloop.remask(st["tokens"], st["conf"], st["in_step"], opos, ocnt)
+            st["remasks"] += 1
+        else:
+            ow, orl, oun = oloop.next_window(st["tokens"], K)
+            assert (d["window"].cpu().numpy() == ow).all() and (d["row_len"].cpu().numpy() == orl).all()
+            assert (d["unresolved"].cpu().numpy() == oun).all()
+            od = oracle.draft_sample(d["q"].cpu(), T, 11, rnd, row_len=orl)
+            used = np.arange(K)[None, :] < orl[:, None]
+            dt = d["draft"].tokens.cpu().numpy()
+            assert (dt[used] == od["tokens"][used]).all()
+            xin = oloop.verification_inputs(st["tokens"], ow, orl, dt)
+            assert (d["inputs"].cpu().numpy() == xin).all()
+            r = d["result"]
+            ref = oracle.spec_verify(d["q"].cpu(), d["p"].cpu(), dt, T, 11, rnd, row_len=orl)
+            ga, gt, gc = r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy()
+            rep = compare_verify(ga, gt, gc, ref)
+            assert rep.ok, rep.mismatches[:5]
+            # the oracle's bookkeeping takes the device's verified values (they agree within the
+            # floating-point tolerance above; the integer work after them must be exact)
+            on = oloop.commit(st["tokens"], st["conf"], st["in_step"], ow, orl, ga, gt, gc)
+            assert (d["committed"].cpu().numpy() == on).all()
+            st["rounds"] += 1
+        assert (d["tokens"].cpu().numpy() == st["tokens"]).all()
+        assert (d["conf"].cpu().numpy() == st["conf"]).all()
+        assert (d["in_step"].cpu().numpy() == st["in_step"]).all()
+
+    out = run_decode_loop_device(fef, B, L, K, 3, 5, logits_fn, T, 11, on_round=on_round, build_inputs=True,
+                                 reuse_draft_norm=(T > 0 and K % 16 == 0))
+    assert (out["tokens"] >= 0).all()
+    assert out["rounds"] == st["rounds"] and st["remasks"] == 2
+    assert sum(out["committed_per_round"]) == B * L + 2 * B * 5

@@ -80,6 +80,57 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key) {
     return ctr;
 }
 
+// The same generator for many counters that differ in their first word only (one batch row,
+// one window position, one call).  The ten round keys come precomputed (kernel-parameter
+// constants, so they cost no instruction), and the parts of rounds one and two that depend on
+// the fixed words alone are worked out once per row.
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+inline PhiloxKeys philox_round_keys(uint64_t seed) {
+    PhiloxKeys k;
+    uint32_t a = static_cast<uint32_t>(seed), b = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        k.k0[r] = a;
+        k.k1[r] = b;
+        a += 0x9E3779B9u;
+        b += 0xBB67AE85u;
+    }
+    return k;
+}
+struct PhiloxRow {
+    uint32_t s1, a1k, c2, d3;
+    __device__ __forceinline__ void prepare(const PhiloxKeys& K, uint32_t c1, uint32_t c2_, uint32_t c3) {
+        constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+        const uint64_t p = static_cast<uint64_t>(M1) * c2_;
+        const uint32_t a0 = static_cast<uint32_t>(p >> 32) ^ c1 ^ K.k0[0];   // word 0 after round one
+        s1 = c3 ^ K.k1[0];
+        a1k = static_cast<uint32_t>(p) ^ K.k0[1];                            // word 1 after round one, keyed
+        const uint64_t q = static_cast<uint64_t>(M0) * a0;
+        c2 = static_cast<uint32_t>(q >> 32) ^ K.k1[1];
+        d3 = static_cast<uint32_t>(q) ^ K.k1[2];                             // word 3 after round two, keyed
+    }
+    __device__ __forceinline__ uint4 draw(const PhiloxKeys& K, uint32_t c0) const {
+        constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+        uint64_t p0 = static_cast<uint64_t>(M0) * c0;                         // round one
+        const uint32_t v2 = static_cast<uint32_t>(p0 >> 32) ^ s1, v3 = static_cast<uint32_t>(p0);
+        uint64_t p1 = static_cast<uint64_t>(M1) * v2;                         // round two
+        const uint32_t w0 = static_cast<uint32_t>(p1 >> 32) ^ a1k, w1 = static_cast<uint32_t>(p1), w2 = v3 ^ c2;
+        p0 = static_cast<uint64_t>(M0) * w0;                                  // round three
+        p1 = static_cast<uint64_t>(M1) * w2;
+        uint4 ctr = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ w1 ^ K.k0[2], static_cast<uint32_t>(p1),
+                               static_cast<uint32_t>(p0 >> 32) ^ d3, static_cast<uint32_t>(p0));
+#pragma unroll
+        for (int r = 3; r < 10; ++r) {
+            p0 = static_cast<uint64_t>(M0) * ctr.x;
+            p1 = static_cast<uint64_t>(M1) * ctr.z;
+            ctr = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ ctr.y ^ K.k0[r], static_cast<uint32_t>(p1),
+                             static_cast<uint32_t>(p0 >> 32) ^ ctr.w ^ K.k1[r], static_cast<uint32_t>(p0));
+        }
+        return ctr;
+    }
+};
+
 // 23 random bits centred in their bin: u in (0, 1), exact in binary32.
 __device__ __forceinline__ float uniform_from_word(uint32_t r) {
     return (static_cast<float>(r >> 9) + 0.5f) * (1.0f / 8388608.0f);

@@ -42,6 +42,7 @@ struct DraftParams {
     float c_hi, c_lo;    // log2(e)/T split in two binary32 numbers (c_lo = 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
+    PhiloxKeys keys;     // round keys of `seed`
     int32_t* tokens;     // [B, K]
     double* log2_norm;   // [B, K] or null
     DraftPart* part_out; // [B*K][parts]
@@ -107,8 +108,9 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
         return;
     }
     const char* lrow = P.logits + row * P.ld_bytes;
-    const uint2 key = make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32));
     const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(i);
+    PhiloxRow rng;
+    rng.prepare(P.keys, ub, upos, P.step);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     RowState st;
@@ -167,8 +169,7 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
 #pragma unroll
                 for (int g4 = 0; g4 < N / 4; ++g4) {
                     const int x0 = vec[j] * N + 4 * g4;
-                    const uint4 r = philox4x32_10(
-                        make_uint4((kStreamDraft << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
+                    const uint4 r = rng.draw(P.keys, (kStreamDraft << 30) | (static_cast<uint32_t>(x0) >> 2));
                     const float t0 = one_minus_uniform(r.x), t1 = one_minus_uniform(r.y);
                     const float t2 = one_minus_uniform(r.z), t3 = one_minus_uniform(r.w);
                     // (a product 0 * inf or a NaN term compares false: -inf logits and bad data never qualify)
@@ -399,6 +400,7 @@ fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len, in
     P.c_hi = c_hi;
     if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
     P.seed = seed;
+    P.keys = philox_round_keys(seed);
     P.step = step;
     P.tokens = draft_tokens;
     P.log2_norm = log2_norm;

@@ -51,6 +51,7 @@ struct VerifyParams {
     float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
+    PhiloxKeys keys;       // round keys of `seed`
     int32_t* accept_len;
     int32_t* tokens;
     float* conf;
@@ -856,8 +857,10 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
     const char* prow = P.target + row * G.ld_bytes;
     const char* qrow = P.draft + row * G.ld_bytes;
     const float kp = static_cast<float>(task.kp), kq = static_cast<float>(task.kq);
-    const uint2 key = make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32));
     const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(task.pos);
+
+    PhiloxRow rng;
+    rng.prepare(P.keys, ub, upos, P.step);
 
     Top2 top;
     top.clear();
@@ -889,6 +892,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
         float floor_w = fmaxf(top.w2, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&s_floor)));
 #pragma unroll
         for (int j = 0; j < kResidualBatch; ++j) {
+            if (v0 + j * kResidualThreads >= v_end) break;  // nothing but padding left (uniform over the CTA)
             float lp[N], lq[N], r[N];
             unpack<DT>(wp[j], lp);
             unpack<DT>(wq[j], lq);
@@ -898,8 +902,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
 #pragma unroll
             for (int g4 = 0; g4 < N / 4; ++g4) {
                 const int x0 = vec[j] * N + 4 * g4;
-                const uint4 w = philox4x32_10(
-                    make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2), ub, upos, P.step), key);
+                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2));
                 // w = r / (-ln u) < r / t: once the floor is up, nearly every id is ruled out by one
                 // multiply and compare; the vote keeps the rare rest out of the straight-line code
                 const float t0 = one_minus_uniform(w.x), t1 = one_minus_uniform(w.y);
@@ -930,8 +933,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
             const float lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
             const float r = exp2_scaled<DT>(lp, P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq, P.c_hi, P.c_lo, kq);
             if (r > 0.f) {
-                const uint4 w = philox4x32_10(
-                    make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), ub, upos, P.step), key);
+                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2));
                 const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
                 top.offer(__fdividef(r, neg_log_uniform(one_minus_uniform(word))), x);
             }
@@ -1250,6 +1252,7 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
     P.row_len = row_len;
     P.draft_norm = greedy ? nullptr : draft_log2_norm;
     P.seed = seed;
+    P.keys = philox_round_keys(seed);
     P.step = step;
     P.accept_len = accept_len;
     P.tokens = tokens;

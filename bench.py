@@ -194,22 +194,15 @@ def run_native(args):
     count = torch.empty(w.B, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
-    call_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
     stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
     for evs in stage_ev:
         for e in evs:
             e.record(stream)  # creates the underlying CUDA event
 
-    def step(i, events=None, stages=None):
+    def step(i, stages=None):
         q, p, tok = sets[i % nbuf]
-        if events:
-            events[0].record(stream)
         fef.fef_spec_verify(q, p, tok, w.temperature, seed, i, out=out, workspace=ws, stage_events=stages)
-        if events:
-            events[1].record(stream)
         fef.fef_remask_select(conf_state, mask_state, w.remask_k, positions=positions, count=count)
-        if events:
-            events[2].record(stream)
 
     def barrier():
         if world > 1:
@@ -229,23 +222,27 @@ def run_native(args):
     t1.record(stream)
     barrier()
     elapsed_ms = t0.elapsed_time(t1)
-    # timed region 2: the same K steps again with CUDA events around each of the two calls, for
-    # the duration of the verification kernel alone (the roofline's kernel)
+    # timed region 2: each of the two calls alone, K times back to back between two CUDA events
+    # (events between the calls would sit inside their dependent-launch chains)
     call_ms = [0.0, 0.0]
     if not args.no_call_events:
+        c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        c0.record(stream)
         for i in range(steps):
-            step(warmup + i, call_ev[i])
+            q, p, tok = sets[(warmup + i) % nbuf]
+            fef.fef_spec_verify(q, p, tok, w.temperature, seed, warmup + i, out=out, workspace=ws)
+        c1.record(stream)
+        for i in range(steps):
+            fef.fef_remask_select(conf_state, mask_state, w.remask_k, positions=positions, count=count)
+        c2.record(stream)
         barrier()
-        for evs in call_ev:
-            for j in range(2):
-                call_ms[j] += evs[j].elapsed_time(evs[j + 1])
-        call_ms = [x / steps for x in call_ms]
+        call_ms = [c0.elapsed_time(c1) / steps, c1.elapsed_time(c2) / steps]
     # timed region 3: once more with events at the kernel boundaries inside the verification call
     # (fef_spec_verify_profiled), for the duration of each kernel alone
     stage_ms = [0.0, 0.0, 0.0]
     if not args.no_call_events:
         for i in range(steps):
-            step(warmup + i, None, stage_ev[i])
+            step(warmup + i, stage_ev[i])
         barrier()
         for evs in stage_ev:
             for j in range(3):
@@ -359,7 +356,7 @@ def run_native(args):
         roof["kernel_ms"] = {"stream_kernel": stage_ms[0], "scan_kernel": stage_ms[1], "residual_kernel": stage_ms[2]}
         roof["timed"] = ("third pass over the same K steps with CUDA events at the kernel boundaries "
                          "(fef_spec_verify_profiled)")
-        # the whole verification call (three kernels chained with dependent launches, two memsets),
+        # the whole verification call (four kernels chained with dependent launches), K calls back to back,
         # every row counted once although the rejected rows are read a second time
         roof["call_ms"] = {"fef_spec_verify": call_ms[0], "fef_remask_select": call_ms[1]}
         roof["call_achieved"] = stream_bytes / (call_ms[0] * 1e-3) / 1e9
@@ -386,7 +383,8 @@ def run_native(args):
                     "by HBM; not part of the step",
             "verify_with_draft_norm_ms": norm_ms,
             "verify_with_draft_norm_positions_per_s": w.B * w.K / (norm_ms * 1e-3)},
-        "gpu_launches": steps * 4,
+        # per step: begin-call, streaming, scan, (sampling mode) residual, re-mask kernels
+        "gpu_launches": steps * (5 if w.temperature > 0 else 4),
         "clocks": sampler.result(),
         "cpu_baseline": cpu_baseline,
         "parity_vs_oracle": parity,

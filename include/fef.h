@@ -11,8 +11,8 @@
  * Conventions
  *  - Pointers marked "device" must be device memory of the current CUDA device;
  *    the caller owns every buffer.  The library allocates nothing, keeps no
- *    state between calls and never synchronises: all work (three kernels per
- *    verification call, preceded by the clearing of a counter) is enqueued on `cuda_stream`
+ *    state between calls and never synchronises: all work (four kernels per
+ *    verification call, the first of which clears a counter and the status word) is enqueued on `cuda_stream`
  *    (a cudaStream_t passed as void*; NULL = the default stream).
  *  - The return value reports what the host can see (bad arguments, launch
  *    failures).  Errors that only the data reveals are written to

@@ -1,7 +1,8 @@
 // fef_spec_verify: the verification loop of the paper's Algorithm 2 for B windows at once.
 //
-// Three kernels, enqueued back to back on the caller's stream (the second and third with
-// programmatic dependent launch):
+// Four kernels, enqueued back to back on the caller's stream and chained with programmatic
+// dependent launch:
+//   begin_call_kernel  one warp: the claim counter and the caller's status word start at zero;
 //   stream_kernel    reads every target and draft row exactly once (bulk-async copies into a
 //                    shared-memory ring; persistent CTAs take runs of tiles, "claims", from a
 //                    shared counter in row order) and leaves, per claim, the partial sum of

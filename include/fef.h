@@ -302,6 +302,36 @@ fef_status fef_loop_commit(const int32_t* window_pos, const int32_t* row_len, co
 fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B, int L, int k,
                            int32_t* tokens, float* conf, uint8_t* in_step, void* cuda_stream);
 
+/*
+ * The same calls with the step number completed on the device, for loops that are replayed as a
+ * CUDA graph (Algorithm 2's "while some position is unresolved" without a host round trip: a
+ * captured round keeps its by-value arguments, so the number that makes every round's random
+ * numbers distinct has to live in device memory).  The step used is step + *device_round, read
+ * when the kernels run.  device_round: device, [1] uint32, required (NULL is
+ * FEF_ERR_INVALID_ARG); it must not change between the draft draws of a round and their
+ * verification.  fef_loop_advance_round adds one to it on `cuda_stream`; when `unresolved`
+ * (device, [B] int32, the output of fef_loop_next_window; may be NULL) is given it does so only
+ * if some row still had an unresolved position, so that replayed rounds with nothing left to
+ * do take no number.
+ * fef_spec_verify_at_round takes draft_log2_norm as fef_spec_verify_with_draft_norm does, or NULL
+ * to stream the draft rows as fef_spec_verify does.  Everything else as in the plain calls.
+ */
+fef_status fef_draft_sample_at_round(const void* draft_logits, const int32_t* row_len,
+                                     int B, int K, int V, int64_t ld, fef_dtype dt,
+                                     float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                     int32_t* draft_tokens, double* log2_norm,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* device_status, void* cuda_stream);
+fef_status fef_spec_verify_at_round(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const double* draft_log2_norm,
+                                    const int32_t* row_len,
+                                    int B, int K, int V, int64_t ld, fef_dtype dt,
+                                    float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                    int32_t* accept_len, int32_t* tokens, float* conf,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* device_status, void* cuda_stream);
+fef_status fef_loop_advance_round(uint32_t* device_round, const int32_t* unresolved, int B, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

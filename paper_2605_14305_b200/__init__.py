@@ -26,7 +26,8 @@ EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_ver
            "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host", "fef_remask_select",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static",
            "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm",
-           "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask")
+           "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask",
+           "fef_draft_sample_at_round", "fef_spec_verify_at_round", "fef_loop_advance_round")
 
 _lib = None
 
@@ -73,6 +74,13 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_draft_sample_workspace_bytes.restype = sz
     L.fef_draft_sample.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.fef_draft_sample.restype = i32
+    L.fef_draft_sample_at_round.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, sz, vp, vp]
+    L.fef_draft_sample_at_round.restype = i32
+    L.fef_spec_verify_at_round.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp,
+                                           vp, sz, vp, vp]
+    L.fef_spec_verify_at_round.restype = i32
+    L.fef_loop_advance_round.argtypes = [vp, vp, i32, vp]
+    L.fef_loop_advance_round.restype = i32
     L.fef_loop_next_window.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     L.fef_loop_verification_inputs.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp]
     L.fef_loop_commit.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -130,7 +138,8 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
                     temperature: float, seed: int, step: int, row_len: Optional[torch.Tensor] = None,
                     V: Optional[int] = None, out: Optional[VerifyResult] = None,
                     workspace: Optional[torch.Tensor] = None, stream=None, stage_events=None,
-                    draft_log2_norm: Optional[torch.Tensor] = None) -> VerifyResult:
+                    draft_log2_norm: Optional[torch.Tensor] = None,
+                    device_round: Optional[torch.Tensor] = None) -> VerifyResult:
     """Enqueue one verification call (see ``fef_spec_verify`` in include/fef.h).
 
     With ``stage_events`` (four ``torch.cuda.Event(enable_timing=True)`` that have
@@ -138,6 +147,8 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
     ``fef_spec_verify_profiled`` and the events mark the kernel boundaries.  With
     ``draft_log2_norm`` (the ``log2_norm`` of ``fef_draft_sample``, ``[B, K]`` float64) the
     call goes through ``fef_spec_verify_with_draft_norm`` and streams the target rows only.
+    With ``device_round`` (a one-element int32 CUDA tensor) the call goes through
+    ``fef_spec_verify_at_round``: the step used is ``step + device_round[0]`` when the kernels run.
 
     ``draft_logits`` / ``target_logits``: ``[B, K, ld]`` CUDA tensors, float32 or
     bfloat16, contiguous; ``V`` (default ``ld``) entries of each row are used.
@@ -172,8 +183,13 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
         if draft_log2_norm is not None:
             if draft_log2_norm.dtype != torch.float64 or draft_log2_norm.numel() != B * K or \
                     not draft_log2_norm.is_contiguous() or draft_log2_norm.device != dev:
-                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm",
-           "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask")
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm")
+        if device_round is not None:
+            if device_round.dtype != torch.int32 or device_round.numel() != 1 or device_round.device != dev:
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_at_round")
+            st = load().fef_spec_verify_at_round(*args[:3], None if draft_log2_norm is None else draft_log2_norm.data_ptr(),
+                                                 *args[3:12], device_round.data_ptr(), *args[12:])
+        elif draft_log2_norm is not None:
             st = load().fef_spec_verify_with_draft_norm(*args[:3], draft_log2_norm.data_ptr(), *args[3:])
         elif stage_events is None:
             st = load().fef_spec_verify(*args)
@@ -199,7 +215,7 @@ def fef_draft_sample_workspace_bytes(B: int, K: int, V: int, dtype) -> int:
 def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, step: int,
                      row_len: Optional[torch.Tensor] = None, V: Optional[int] = None,
                      out: Optional[DraftResult] = None, workspace: Optional[torch.Tensor] = None,
-                     stream=None) -> DraftResult:
+                     stream=None, device_round: Optional[torch.Tensor] = None) -> DraftResult:
     """Enqueue the draft-token draws of one call (see ``fef_draft_sample`` in include/fef.h).
 
     ``draft_logits``: ``[B, K, ld]`` CUDA tensor, float32 or bfloat16, contiguous; ``V`` (default
@@ -222,11 +238,16 @@ def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, 
         if workspace is None:
             workspace = torch.empty(max(fef_draft_sample_workspace_bytes(B, K, V, code), 256), dtype=torch.uint8,
                                     device=dev)
-        st = load().fef_draft_sample(draft_logits.data_ptr(), None if row_len is None else row_len.data_ptr(),
-                                     B, K, V, ld, code, float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF,
-                                     int(step) & 0xFFFFFFFF, out.tokens.data_ptr(), out.log2_norm.data_ptr(),
-                                     workspace.data_ptr(), workspace.numel(), out.device_status.data_ptr(),
-                                     _stream_ptr(stream))
+        head = (draft_logits.data_ptr(), None if row_len is None else row_len.data_ptr(), B, K, V, ld, code,
+                float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF)
+        tail = (out.tokens.data_ptr(), out.log2_norm.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                out.device_status.data_ptr(), _stream_ptr(stream))
+        if device_round is None:
+            st = load().fef_draft_sample(*head, *tail)
+        else:
+            if device_round.dtype != torch.int32 or device_round.numel() != 1 or device_round.device != dev:
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_draft_sample_at_round")
+            st = load().fef_draft_sample_at_round(*head, device_round.data_ptr(), *tail)
     if st != FEF_OK:
         raise FefError(st, "fef_draft_sample")
     return out
@@ -286,6 +307,20 @@ def fef_loop_commit(window_pos, row_len, verified: "VerifyResult", tokens, conf,
     if st != FEF_OK:
         raise FefError(st, "fef_loop_commit")
     return committed
+
+
+def fef_loop_advance_round(device_round: torch.Tensor, unresolved: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Add one to the device-resident round counter (a one-element int32 CUDA tensor); with
+    ``unresolved`` (``[B]`` int32, from ``fef_loop_next_window``) only if some row had work left."""
+    _i32_cuda(device_round, "fef_loop_advance_round")
+    if unresolved is not None:
+        _i32_cuda(unresolved, "fef_loop_advance_round")
+    with torch.cuda.device(device_round.device):
+        st = load().fef_loop_advance_round(device_round.data_ptr(),
+                                           None if unresolved is None else unresolved.data_ptr(),
+                                           0 if unresolved is None else unresolved.numel(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_advance_round")
 
 
 def fef_loop_remask(positions, count, tokens, conf, in_step, stream=None) -> None:
@@ -434,7 +469,7 @@ def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena
     return positions, count
 
 
-__all__ = ["fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask", "MASK_TOKEN",
+__all__ = ["fef_loop_advance_round", "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask", "MASK_TOKEN",
            "fef_draft_sample", "fef_draft_sample_workspace_bytes", "DraftResult", "fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]

@@ -42,6 +42,7 @@ struct DraftParams {
     float c_hi, c_lo;    // log2(e)/T split in two binary32 numbers (c_lo = 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
+    const uint32_t* round; // device word added to `step` when the kernel runs, or null
     PhiloxKeys keys;     // round keys of `seed`
     int32_t* tokens;     // [B, K]
     double* log2_norm;   // [B, K] or null
@@ -80,12 +81,16 @@ struct BestTwo {
     }
 };
 
+__device__ __forceinline__ uint32_t step_of(const DraftParams& P) {
+    return P.step + (P.round ? __ldg(P.round) : 0u);
+}
+
 // Exact (double) key l / T - ln(-ln u) of vocabulary id x, in units of log2: l c - log2(-ln u).
 template <int DT>
 __device__ double exact_key(int x, const char* row, double c, uint32_t b, uint32_t pos, const DraftParams& P) {
     const double l = load_logit<DT>(row, x);
     if (!(l > -INFINITY)) return -INFINITY;
-    const uint4 w = philox4x32_10(make_uint4((kStreamDraft << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, P.step),
+    const uint4 w = philox4x32_10(make_uint4((kStreamDraft << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, step_of(P)),
                                   make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
     const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
     const double u = uniform_from_word(word);
@@ -110,7 +115,7 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
     const char* lrow = P.logits + row * P.ld_bytes;
     const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(i);
     PhiloxRow rng;
-    rng.prepare(P.keys, ub, upos, P.step);
+    rng.prepare(P.keys, ub, upos, step_of(P));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     RowState st;
@@ -359,10 +364,12 @@ size_t fef_draft_sample_workspace_bytes(int B, int K, int V, fef_dtype dt) {
            fef::draft_round256(rows * fef::kDraftMaxParts * sizeof(fef::DraftPart));
 }
 
-fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
-                            fef_dtype dt, float temperature, uint64_t seed, uint32_t step, int32_t* draft_tokens,
-                            double* log2_norm, void* workspace, size_t workspace_bytes, int32_t* device_status,
-                            void* cuda_stream) {
+}  // extern "C"
+
+static fef_status draft_impl(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
+                             fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                             const uint32_t* device_round, int32_t* draft_tokens, double* log2_norm, void* workspace,
+                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !draft_tokens) return FEF_ERR_INVALID_ARG;
@@ -402,6 +409,7 @@ fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len, in
     P.seed = seed;
     P.keys = philox_round_keys(seed);
     P.step = step;
+    P.round = device_round;
     P.tokens = draft_tokens;
     P.log2_norm = log2_norm;
     const size_t rows = static_cast<size_t>(B) * K;
@@ -427,6 +435,26 @@ fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len, in
             draft_kernel<FEF_BF16, false><<<grid, kDraftThreads, 0, stream>>>(P);
     }
     return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+extern "C" {
+
+fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
+                            fef_dtype dt, float temperature, uint64_t seed, uint32_t step, int32_t* draft_tokens,
+                            double* log2_norm, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                            void* cuda_stream) {
+    return draft_impl(draft_logits, row_len, B, K, V, ld, dt, temperature, seed, step, nullptr, draft_tokens, log2_norm,
+                      workspace, workspace_bytes, device_status, cuda_stream);
+}
+
+fef_status fef_draft_sample_at_round(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
+                                     fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                                     const uint32_t* device_round, int32_t* draft_tokens, double* log2_norm,
+                                     void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                     void* cuda_stream) {
+    if (!device_round) return FEF_ERR_INVALID_ARG;
+    return draft_impl(draft_logits, row_len, B, K, V, ld, dt, temperature, seed, step, device_round, draft_tokens,
+                      log2_norm, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
 }  // extern "C"

@@ -106,6 +106,17 @@ __global__ void remask_apply_kernel(const int32_t* __restrict__ positions, const
     }
 }
 
+// The round counter that fef_draft_sample_at_round / fef_spec_verify_at_round read: plus one,
+// unless `unresolved` is given and no row has an unresolved position left (a replayed round
+// that had nothing to do takes no number).
+__global__ void __launch_bounds__(kLoopThreads) advance_round_kernel(uint32_t* round, const int32_t* unresolved, int B) {
+    int any = unresolved ? 0 : 1;
+    if (unresolved)
+        for (int b = threadIdx.x; b < B; b += kLoopThreads) any |= unresolved[b] > 0;
+    any = __syncthreads_or(any);
+    if (threadIdx.x == 0 && any) *round += 1u;
+}
+
 static bool loop_sizes_ok(int B, int L, int K) {
     return B >= 1 && B <= FEF_MAX_B && L >= 1 && L <= (1 << 24) && K >= 1 && K <= FEF_MAX_K;
 }
@@ -154,6 +165,13 @@ fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B
         return FEF_ERR_INVALID_ARG;
     remask_apply_kernel<<<B, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(positions, count, L, k, tokens, conf,
                                                                               in_step);
+    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_loop_advance_round(uint32_t* device_round, const int32_t* unresolved, int B, void* cuda_stream) {
+    if (!device_round || (unresolved && (B < 1 || B > FEF_MAX_B))) return FEF_ERR_INVALID_ARG;
+    fef::advance_round_kernel<<<1, fef::kLoopThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(device_round,
+                                                                                                 unresolved, B);
     return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 

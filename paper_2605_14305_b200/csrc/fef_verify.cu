@@ -52,6 +52,7 @@ struct VerifyParams {
     float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
     uint64_t seed;
     uint32_t step;
+    const uint32_t* round; // device word added to `step` when the kernels run, or null
     PhiloxKeys keys;       // round keys of `seed`
     int32_t* accept_len;
     int32_t* tokens;
@@ -62,6 +63,12 @@ struct VerifyParams {
     Candidate* candidates; // [B][residual_ctas][2]
     int32_t* status;
 };
+
+// The call's step number: the by-value part plus, if given, a device-resident round counter
+// (read when the kernel runs, so that a replayed CUDA graph draws fresh random numbers).
+__device__ __forceinline__ uint32_t step_of(const VerifyParams& P) {
+    return P.step + (P.round ? __ldg(P.round) : 0u);
+}
 
 // ============================================================ streaming ====
 // One 16-byte vector, packed two-wide binary32 arithmetic (fma.rn.f32x2 / add.f32x2):
@@ -551,7 +558,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
                     } else {
                         const double ratio = exp2(l2pi - (lqx[r] * c - kq[r]));
                         const uint4 rnd = philox4x32_10(
-                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), P.step),
+                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
                             make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
                         const double uacc = uniform_from_word(rnd.x);
                         accept = uacc <= fmin(1.0, ratio);
@@ -754,7 +761,7 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
                     } else {
                         const double ratio = exp2(l2pi - (lqx * c - kq));
                         const uint4 r = philox4x32_10(
-                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), P.step),
+                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
                             make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
                         const double uacc = uniform_from_word(r.x);
                         accept = uacc <= fmin(1.0, ratio);
@@ -822,7 +829,7 @@ __device__ double exact_score(int x, const char* prow, const char* qrow, double 
     const double r = pi - rho;
     if (!(r > 0.0)) return -INFINITY;
     const uint4 w = philox4x32_10(
-        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, P.step),
+        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, step_of(P)),
         make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
     const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
     const double u = uniform_from_word(word);
@@ -872,7 +879,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
     const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(task.pos);
 
     PhiloxRow rng;
-    rng.prepare(P.keys, ub, upos, P.step);
+    rng.prepare(P.keys, ub, upos, step_of(P));
 
     Top2 top;
     top.clear();
@@ -1230,7 +1237,8 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
                               const int32_t* row_len, const double* draft_log2_norm, int B, int K, int V, int64_t ld,
                               fef_dtype dt, float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
                               int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
-                              int32_t* device_status, void* cuda_stream, void* const* stage_events) {
+                              int32_t* device_status, void* cuda_stream, void* const* stage_events,
+                              const uint32_t* device_round = nullptr) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -1277,6 +1285,7 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
     P.seed = seed;
     P.keys = philox_round_keys(seed);
     P.step = step;
+    P.round = device_round;
     P.accept_len = accept_len;
     P.tokens = tokens;
     P.conf = conf;
@@ -1332,6 +1341,18 @@ fef_status fef_spec_verify_with_draft_norm(const void* draft_logits, const void*
     return verify_impl(draft_logits, target_logits, draft_tokens, row_len, draft_log2_norm, B, K, V, ld, dt,
                        temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes, device_status,
                        cuda_stream, nullptr);
+}
+
+fef_status fef_spec_verify_at_round(const void* draft_logits, const void* target_logits,
+                                    const int32_t* draft_tokens, const double* draft_log2_norm,
+                                    const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                                    float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                    int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
+                                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    if (!device_round) return FEF_ERR_INVALID_ARG;
+    return verify_impl(draft_logits, target_logits, draft_tokens, row_len, draft_log2_norm, B, K, V, ld, dt,
+                       temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes, device_status,
+                       cuda_stream, nullptr, device_round);
 }
 
 // ---- host-buffer variant: layout of the caller's device arena

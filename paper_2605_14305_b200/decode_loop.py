@@ -136,3 +136,63 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
                 on_round(None, dict(positions=positions, count=count, before=before,
                                     tokens=tokens, conf=conf, in_step=in_step))
     return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist)
+
+
+def run_decode_loop_graph(fef, B: int, L: int, K: int, n_steps: int, remask_k: int, logits_fn: Callable,
+                          temperature: float, seed: int, first_round: int = 0, reuse_draft_norm: bool = True,
+                          rounds_per_check: int = 4):
+    """``run_decode_loop_device`` with one whole round captured as a CUDA graph and replayed.
+
+    The round's number lives in a device word that ``fef_draft_sample`` / ``fef_spec_verify`` add
+    to their step (``device_round=``) and ``fef_loop_advance_round`` bumps while some row still
+    has unresolved positions, so every replay draws the random numbers the eager loop would.  The
+    host launches ``rounds_per_check`` replays at a time and then reads one integer; replays after
+    the last real round of a denoising step change nothing.
+
+    logits_fn(device_round [1] int32 CUDA, window_pos, row_len) -> (draft_logits, target_logits):
+    must be capturable (device work only, the round read from the tensor).
+
+    Returns dict(tokens, conf (CUDA), rounds).
+    """
+    dev = torch.device("cuda")
+    tokens = torch.full((B, L), MASK, dtype=torch.int32, device=dev)
+    conf = torch.full((B, L), -1.0, dtype=torch.float32, device=dev)
+    in_step = torch.zeros((B, L), dtype=torch.uint8, device=dev)
+    rnd = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def one_round():
+        window, row_len, unresolved = fef.fef_loop_next_window(tokens, K)
+        q, p = logits_fn(rnd, window, row_len)
+        draft = fef.fef_draft_sample(q, temperature, seed, first_round, row_len=row_len, device_round=rnd)
+        res = fef.fef_spec_verify(q, p, draft.tokens, temperature, seed, first_round, row_len=row_len,
+                                  draft_log2_norm=draft.log2_norm if reuse_draft_norm else None, device_round=rnd)
+        fef.fef_loop_commit(window, row_len, res, tokens, conf, in_step)
+        fef.fef_loop_advance_round(rnd, unresolved)
+        return unresolved
+
+    # one eager round on a side stream first (per-device set-up of the library, allocator warm-up),
+    # then the state is put back and the same round is captured
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        one_round()
+    torch.cuda.current_stream().wait_stream(side)
+    tokens.fill_(MASK)
+    conf.fill_(-1.0)
+    in_step.zero_()
+    rnd.zero_()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        unresolved = one_round()
+
+    for s in range(n_steps):
+        while True:
+            for _ in range(rounds_per_check):
+                graph.replay()
+            if int(unresolved.max().item()) == 0:   # counted before the last replay: nothing was left
+                break
+        if s < n_steps - 1 and remask_k > 0:
+            positions, count = fef.fef_remask_select(conf, in_step, remask_k)
+            fef.fef_loop_remask(positions, count, tokens, conf, in_step)
+    return dict(tokens=tokens, conf=conf, rounds=int(rnd.item()))

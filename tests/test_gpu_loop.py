@@ -144,3 +144,56 @@ def test_device_resident_loop_matches_the_oracle_round_by_round(fef, B, K, L, dt
     assert (out["tokens"] >= 0).all()
     assert out["rounds"] == st["rounds"] and st["remasks"] == 2
     assert sum(out["committed_per_round"]) == B * L + 2 * B * 5
+
+
+def test_at_round_entry_points_equal_the_plain_calls_at_the_summed_step(fef):
+    """step + *device_round is the step: same draws, same verification, bit for bit."""
+    w = synth.TINY.with_(B=3, K=8, V=4096, dtype=torch.bfloat16, noise_std=0.6)
+    q, p = synth.make_logits(w, seed=5, device="cuda")
+    rnd = torch.tensor([37], dtype=torch.int32, device="cuda")
+    d0 = fef.fef_draft_sample(q, 1.0, 9, 100 + 37)
+    d1 = fef.fef_draft_sample(q, 1.0, 9, 100, device_round=rnd)
+    assert (d0.tokens == d1.tokens).all() and (d0.log2_norm == d1.log2_norm).all()
+    for norm in (None, d0.log2_norm):
+        r0 = fef.fef_spec_verify(q, p, d0.tokens, 1.0, 9, 137, draft_log2_norm=norm)
+        r1 = fef.fef_spec_verify(q, p, d0.tokens, 1.0, 9, 100, draft_log2_norm=norm, device_round=rnd)
+        assert (r0.accept_len == r1.accept_len).all() and (r0.tokens == r1.tokens).all() and (r0.conf == r1.conf).all()
+    ref = oracle.spec_verify(q.cpu(), p.cpu(), d0.tokens.cpu(), 1.0, 9, 137)
+    r1 = fef.fef_spec_verify(q, p, d0.tokens, 1.0, 9, 100, device_round=rnd)
+    rep = compare_verify(r1.accept_len.cpu().numpy(), r1.tokens.cpu().numpy(), r1.conf.cpu().numpy(), ref)
+    assert rep.ok, rep.mismatches[:5]
+    # the counter moves only while some row has work left
+    un = torch.tensor([0, 0, 0], dtype=torch.int32, device="cuda")
+    fef.fef_loop_advance_round(rnd, un)
+    assert int(rnd.item()) == 37
+    un[1] = 2
+    fef.fef_loop_advance_round(rnd, un)
+    fef.fef_loop_advance_round(rnd)
+    assert int(rnd.item()) == 39
+
+
+@pytest.mark.parametrize("B,K,L,dtype,norm", [(2, 4, 40, torch.float32, False), (4, 8, 96, torch.bfloat16, True)])
+def test_replayed_graph_of_a_round_equals_the_eager_device_loop(fef, B, K, L, dtype, norm):
+    """One round captured as a CUDA graph and replayed (round number on the device) against the
+    eager device-resident loop, which the test above checks against the oracle round by round."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device, run_decode_loop_graph
+
+    w = synth.TINY.with_(B=B, K=K, V=2048, dtype=dtype, noise_std=0.6)
+    R = 16
+    pool = [synth.make_logits(w, seed=900 + r, device="cuda") for r in range(R)]
+    pool_q = torch.stack([x[0] for x in pool])
+    pool_p = torch.stack([x[1] for x in pool])
+
+    def eager_logits(rnd, window, row_len, inputs):
+        return pool_q[rnd % R], pool_p[rnd % R]
+
+    def graph_logits(device_round, window, row_len):
+        idx = torch.remainder(device_round, R).to(torch.int64)
+        return pool_q.index_select(0, idx)[0], pool_p.index_select(0, idx)[0]
+
+    a = run_decode_loop_device(fef, B, L, K, 3, 4, eager_logits, 1.0, 21, reuse_draft_norm=norm)
+    g = run_decode_loop_graph(fef, B, L, K, 3, 4, graph_logits, 1.0, 21, reuse_draft_norm=norm)
+    torch.cuda.synchronize()
+    assert g["rounds"] == a["rounds"]
+    assert (g["tokens"] == a["tokens"]).all() and (g["conf"] == a["conf"]).all()
+    assert (g["tokens"] >= 0).all()

@@ -19,6 +19,7 @@ same driver can run any implementation.
 """
 from __future__ import annotations
 
+import time
 from typing import Callable, Optional
 
 import numpy as np
@@ -96,7 +97,7 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
     on_round(round, dict of the round's device tensors): optional hook, called after the commit with
     the state before it under "before"; called with round None after each re-masking.
 
-    Returns dict(tokens [B,L] int32, conf [B,L] float32 (CUDA), rounds, committed_per_round).
+    Returns dict(tokens [B,L] int32, conf [B,L] float32 (CUDA), rounds, committed_per_round, loop_seconds).
     """
     dev = torch.device("cuda")
     tokens = torch.full((B, L), MASK, dtype=torch.int32, device=dev)
@@ -104,6 +105,8 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
     in_step = torch.zeros((B, L), dtype=torch.uint8, device=dev)
     rnd = first_round
     committed_hist = []
+    torch.cuda.synchronize()
+    t_start = time.perf_counter()
     for s in range(n_steps):
         while True:
             window, row_len, unresolved = fef.fef_loop_next_window(tokens, K)
@@ -135,7 +138,9 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
             if on_round is not None:
                 on_round(None, dict(positions=positions, count=count, before=before,
                                     tokens=tokens, conf=conf, in_step=in_step))
-    return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist)
+    torch.cuda.synchronize()
+    return dict(tokens=tokens, conf=conf, rounds=rnd - first_round, committed_per_round=committed_hist,
+                loop_seconds=time.perf_counter() - t_start)
 
 
 def run_decode_loop_graph(fef, B: int, L: int, K: int, n_steps: int, remask_k: int, logits_fn: Callable,
@@ -152,7 +157,7 @@ def run_decode_loop_graph(fef, B: int, L: int, K: int, n_steps: int, remask_k: i
     logits_fn(device_round [1] int32 CUDA, window_pos, row_len) -> (draft_logits, target_logits):
     must be capturable (device work only, the round read from the tensor).
 
-    Returns dict(tokens, conf (CUDA), rounds).
+    Returns dict(tokens, conf (CUDA), rounds, loop_seconds: wall time of the replay loop alone).
     """
     dev = torch.device("cuda")
     tokens = torch.full((B, L), MASK, dtype=torch.int32, device=dev)
@@ -186,6 +191,8 @@ def run_decode_loop_graph(fef, B: int, L: int, K: int, n_steps: int, remask_k: i
     with torch.cuda.graph(graph):
         unresolved = one_round()
 
+    torch.cuda.synchronize()
+    t_start = time.perf_counter()
     for s in range(n_steps):
         while True:
             for _ in range(rounds_per_check):
@@ -195,4 +202,5 @@ def run_decode_loop_graph(fef, B: int, L: int, K: int, n_steps: int, remask_k: i
         if s < n_steps - 1 and remask_k > 0:
             positions, count = fef.fef_remask_select(conf, in_step, remask_k)
             fef.fef_loop_remask(positions, count, tokens, conf, in_step)
-    return dict(tokens=tokens, conf=conf, rounds=int(rnd.item()))
+    torch.cuda.synchronize()
+    return dict(tokens=tokens, conf=conf, rounds=int(rnd.item()), loop_seconds=time.perf_counter() - t_start)

@@ -12,9 +12,11 @@ namespace fef {
 constexpr int kConsumerWarps = 16;                      // warps that do arithmetic in the streaming kernel
 constexpr int kProducerWarp = kConsumerWarps;           // one thread of it feeds the ring
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
-constexpr int kVecPerThread = 4;                        // 16-byte vectors per thread per tile
-constexpr int kTileBytes = kConsumerWarps * 32 * 16 * kVecPerThread;  // 32 KiB
-constexpr int kStages = 5;                              // ring depth: 160 KiB in flight per SM
+constexpr int kVecPerThread = 4;                        // 16-byte vectors per thread per chunk
+constexpr int kChunkBytes = kConsumerWarps * 32 * 16 * kVecPerThread;  // 32 KiB: what the consumers take in one go
+constexpr int kHalves = 2;                              // chunks per tile: one barrier wait and one release per 64 KiB
+constexpr int kTileBytes = kChunkBytes * kHalves;       // 64 KiB
+constexpr int kStages = 3;                              // ring depth: 192 KiB in flight per SM
 constexpr int kSpinLimit = 1 << 22;                     // bound on every mbarrier wait loop
 constexpr int kSlotSets = 8;                            // in-CTA combine buffers (a warp leads by < 8 flushes)
 

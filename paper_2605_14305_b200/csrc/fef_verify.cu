@@ -29,7 +29,7 @@ struct Geometry {
     int B, K, V;
     int units_per_row;    // 2: target row and draft row; 1 when only the target rows are streamed (greedy
                           // mode, or the draft laws' normalisers are given)
-    int tile_bytes;       // bytes of one streaming tile (8, 16 or 32 KiB)
+    int tile_bytes;       // bytes of one streaming tile (8, 16, 32 or 64 KiB)
     int vec_bytes;        // bytes of a row covered by whole 16-byte vectors
     int vec_elems;        // the same in elements; elements beyond are the row's "tail"
     int tiles_per_unit;   // tiles per row (0 when a row holds no whole vector)
@@ -334,36 +334,45 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             const unsigned char* stage = smem + s * kTileBytes;
 
             if (d.flags & kFlagFirst) st.reset();
-            uint4 w[kVecPerThread];
-            int at[kVecPerThread];
-#pragma unroll
-            for (int j = 0; j < kVecPerThread; ++j) {
-                at[j] = ((j * kConsumerWarps + warp) * 32 + lane) * 16;
-                if (at[j] < d.len) w[j] = *reinterpret_cast<const uint4*>(stage + at[j]);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty + s);  // the stage may be refilled
+            const int s_cur = s;
             if (++s == kStages) {
                 s = 0;
                 phase ^= 1u;
             }
-            if (d.len > 0) {
-                if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
-                float tile_sum;
-                if (d.len == kTileBytes)  // branch-free: the four vectors interleave
-                    tile_sum = absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
-                else
-                    tile_sum = absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
-                if constexpr (GREEDY) {
-                    const float floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
-                    // 0.999: the sum and the bound carry a few units of 1e-7 of rounding each
-                    const bool candidate = !(tile_sum < 0.999f * exp2_scaled<DT>(floor_f, P.c_hi, P.c_lo, st.ref));
-                    if (__any_sync(0xFFFFFFFFu, candidate)) {  // the vote keeps this out of the straight-line code
-                        if (candidate) {
+            // a tile is taken in chunks of kVecPerThread vectors per thread: the wait, the descriptor
+            // and the release are paid once per tile, the registers hold one chunk
 #pragma unroll
-                            for (int j = 0; j < kVecPerThread; ++j)
-                                if (at[j] < d.len)
-                                    track_best<DT>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, st);
+            for (int h = 0; h < kHalves; ++h) {
+                const int hbase = h * kChunkBytes;
+                uint4 w[kVecPerThread];
+                int at[kVecPerThread];
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    at[j] = hbase + ((j * kConsumerWarps + warp) * 32 + lane) * 16;
+                    if (at[j] < d.len) w[j] = *reinterpret_cast<const uint4*>(stage + at[j]);
+                }
+                if (h == kHalves - 1) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty + s_cur);  // the stage may be refilled
+                }
+                if (d.len > hbase) {
+                    if (st.ref == kNoReference && at[0] < d.len) st.ref = first_reference<DT>(w[0], P.c_hi, P.c_lo);
+                    float tile_sum;
+                    if (d.len >= hbase + kChunkBytes)  // branch-free: the four vectors interleave
+                        tile_sum = absorb_tile<DT, true>(w, at, d.len, P.c_hi, P.c_lo, st);
+                    else
+                        tile_sum = absorb_tile<DT, false>(w, at, d.len, P.c_hi, P.c_lo, st);
+                    if constexpr (GREEDY) {
+                        const float floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
+                        // 0.999: the sum and the bound carry a few units of 1e-7 of rounding each
+                        const bool candidate = !(tile_sum < 0.999f * exp2_scaled<DT>(floor_f, P.c_hi, P.c_lo, st.ref));
+                        if (__any_sync(0xFFFFFFFFu, candidate)) {  // the vote keeps this out of the straight-line code
+                            if (candidate) {
+#pragma unroll
+                                for (int j = 0; j < kVecPerThread; ++j)
+                                    if (at[j] < d.len)
+                                        track_best<DT>(w[j], (d.offset + at[j]) / Elem<DT>::kBytes, st);
+                            }
                         }
                     }
                 }

@@ -332,6 +332,60 @@ fef_status fef_spec_verify_at_round(const void* draft_logits, const void* target
                                     int32_t* device_status, void* cuda_stream);
 fef_status fef_loop_advance_round(uint32_t* device_round, const int32_t* unresolved, int B, void* cuda_stream);
 
+/*
+ * Vocabulary-parallel verification: fef_spec_verify (Algorithm 2's verification loop, the laws of
+ * Section 3.2, the residual law defined before Algorithm 2) when each of `ranks` GPUs holds a
+ * slice [vocab_offset, vocab_offset + V_local) of every logit row, as logits leave a
+ * tensor-parallel output layer.  Sampling mode only (temperature > 0).  The library does the
+ * per-rank work; the caller moves the two small messages between ranks (an all-gather each):
+ *
+ *   1. fef_vp_local_stats     streams this rank's slices once and writes, per position, six
+ *                             doubles: reference and sum of both laws over the slice, and the two
+ *                             logits at the draft token on the rank that holds it (NaN elsewhere).
+ *                             stats: device out, [B*K][6] float64.
+ *      -> all-gather to stats_all [ranks][B*K][6]
+ *   2. fef_vp_accept          folds the ranks' numbers into pi_i(x_i), rho_i(x_i), applies the
+ *                             acceptance tests (same random numbers as fef_spec_verify) and writes
+ *                             accept_len, the accepted tokens and confidences, and per window the
+ *                             rejected position with its normalisers (`tasks`, device, opaque,
+ *                             fef_vp_task_bytes(B) bytes).  Every rank computes the same.
+ *   3. fef_vp_local_residual  Gumbel-max over this rank's slice of every rejected row with the
+ *                             global ids' random numbers; writes its best candidate per window.
+ *                             candidates: device out, [B] records of 16 bytes (float64 score,
+ *                             float32 target logit, int32 global id); windows without a rejection
+ *                             are left untouched.
+ *      -> all-gather to candidates_all [ranks][B]
+ *   4. fef_vp_finish          largest score wins (lowest id on ties; if [pi - rho]_+ is zero
+ *                             everywhere, the largest target logit): writes tokens[b, a_b] and
+ *                             conf[b, a_b].
+ *
+ * Results equal fef_spec_verify's on the concatenated rows up to the rounding order of the sums.
+ * vocab_offset must be a multiple of 8; slices must tile [0, V_total) without overlap; workspace:
+ * fef_spec_verify_workspace_bytes(B, K, V_local, dt) bytes per rank, shared by steps 1 and 3.
+ * Arguments not listed are as in fef_spec_verify; step 1 needs neither seed nor step.
+ */
+size_t fef_vp_task_bytes(int B);
+fef_status fef_vp_local_stats(const void* draft_slice, const void* target_slice,
+                              const int32_t* draft_tokens, const int32_t* row_len,
+                              int B, int K, int V_local, int64_t ld, fef_dtype dt,
+                              float temperature, int vocab_offset, double* stats,
+                              void* workspace, size_t workspace_bytes,
+                              int32_t* device_status, void* cuda_stream);
+fef_status fef_vp_accept(const double* stats_all, int ranks,
+                         const int32_t* draft_tokens, const int32_t* row_len,
+                         int B, int K, int V_total, fef_dtype dt,
+                         float temperature, uint64_t seed, uint32_t step,
+                         int32_t* accept_len, int32_t* tokens, float* conf, void* tasks,
+                         int32_t* device_status, void* cuda_stream);
+fef_status fef_vp_local_residual(const void* draft_slice, const void* target_slice, void* tasks,
+                                 int B, int K, int V_local, int64_t ld, fef_dtype dt,
+                                 float temperature, uint64_t seed, uint32_t step, int vocab_offset,
+                                 void* candidates, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream);
+fef_status fef_vp_finish(const void* candidates_all, int ranks, const void* tasks,
+                         int B, int K, fef_dtype dt, float temperature,
+                         int32_t* tokens, float* conf, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,8 @@ EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_ver
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host", "fef_spec_verify_static",
            "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm",
            "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask",
-           "fef_draft_sample_at_round", "fef_spec_verify_at_round", "fef_loop_advance_round")
+           "fef_draft_sample_at_round", "fef_spec_verify_at_round", "fef_loop_advance_round",
+           "fef_vp_task_bytes", "fef_vp_local_stats", "fef_vp_accept", "fef_vp_local_residual", "fef_vp_finish")
 
 _lib = None
 
@@ -81,6 +82,16 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_at_round.restype = i32
     L.fef_loop_advance_round.argtypes = [vp, vp, i32, vp]
     L.fef_loop_advance_round.restype = i32
+    L.fef_vp_task_bytes.argtypes = [i32]
+    L.fef_vp_task_bytes.restype = sz
+    L.fef_vp_local_stats.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, i32, vp, vp, sz, vp, vp]
+    L.fef_vp_local_stats.restype = i32
+    L.fef_vp_accept.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp, vp, vp]
+    L.fef_vp_accept.restype = i32
+    L.fef_vp_local_residual.argtypes = [vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, i32, vp, vp, sz, vp]
+    L.fef_vp_local_residual.restype = i32
+    L.fef_vp_finish.argtypes = [vp, i32, vp, i32, i32, i32, f32, vp, vp, vp]
+    L.fef_vp_finish.restype = i32
     L.fef_loop_next_window.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     L.fef_loop_verification_inputs.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp]
     L.fef_loop_commit.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]

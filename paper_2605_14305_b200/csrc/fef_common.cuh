@@ -48,6 +48,14 @@ struct __align__(16) Control {
     unsigned long long next_claim;  // next streaming claim to hand out
 };
 
+// Vocabulary-parallel verification: what one rank reports for a rejected window after its
+// share of the residual draw.
+struct __align__(16) VpCandidate {
+    double score;  // exact Gumbel score ln r - ln(-ln u) of the rank's best id, -inf if its slice has no r > 0
+    float lp;      // target logit of `index`
+    int index;     // global vocabulary id: the best id, or (score = -inf) the slice's arg-max of the target logits
+};
+
 struct __align__(8) Candidate {
     float w;  // r_x / (-ln u_x) in binary32, <= 0 when empty
     int x;

@@ -61,6 +61,8 @@ struct VerifyParams {
     Partial* partials;     // [num_claims]: unit u owns entries [u * claims_per_unit, ...)
     ResidualTask* tasks;   // [B]
     Candidate* candidates; // [B][residual_ctas][2]
+    int vocab_offset;      // global id of element 0 of every row (a multiple of 8; 0 unless the vocabulary is sharded)
+    VpCandidate* vp_out;   // [B] vocabulary-parallel mode: the residual kernel reports here instead of committing
     int32_t* status;
 };
 
@@ -429,6 +431,7 @@ struct RowNorm {
     float best;   // greedy: largest logit
     int index;    // greedy: its lowest index
     bool bad;
+    bool data_bad; // a NaN or +inf was seen (bad also covers rows without any finite logit)
 };
 
 // Fold the claims' partials of unit u (and the row's tail elements, which the streaming
@@ -482,6 +485,7 @@ __device__ __forceinline__ RowNorm fold_unit(int64_t u, const char* row, double 
     out.best = best;
     out.index = index;
     out.bad = bad || !(sacc > 0.0) || !(sacc < INFINITY);
+    out.data_bad = bad || !(sacc < INFINITY) || sacc != sacc;
     return out;
 }
 
@@ -707,6 +711,7 @@ __device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const Ve
     out.best = best;
     out.index = index;
     out.bad = bad || !(S > 0.0) || !(S < INFINITY);
+    out.data_bad = bad || !(S < INFINITY) || S != S;
     return out;
 }
 
@@ -838,7 +843,7 @@ __device__ double exact_score(int x, const char* prow, const char* qrow, double 
     const double r = pi - rho;
     if (!(r > 0.0)) return -INFINITY;
     const uint4 w = philox4x32_10(
-        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2), b, pos, step_of(P)),
+        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x + P.vocab_offset) >> 2), b, pos, step_of(P)),
         make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
     const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
     const double u = uniform_from_word(word);
@@ -930,7 +935,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
 #pragma unroll
             for (int g4 = 0; g4 < N / 4; ++g4) {
                 const int x0 = vec[j] * N + 4 * g4;
-                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x0) >> 2));
+                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x0 + P.vocab_offset) >> 2));
                 // w = r / (-ln u) < r / t: once the floor is up, nearly every id is ruled out by one
                 // multiply and compare; the vote keeps the rare rest out of the straight-line code
                 const float t0 = one_minus_uniform(w.x), t1 = one_minus_uniform(w.y);
@@ -961,7 +966,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
             const float lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
             const float r = exp2_scaled<DT>(lp, P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq, P.c_hi, P.c_lo, kq);
             if (r > 0.f) {
-                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x) >> 2));
+                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x + P.vocab_offset) >> 2));
                 const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
                 top.offer(__fdividef(r, neg_log_uniform(one_minus_uniform(word))), x);
             }
@@ -1017,6 +1022,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
     }
     block_argmax(score, Z, s_score, s_x);
 
+    bool have_score = true;
     if (!(score > -INFINITY)) {
         // Nothing survived in binary32 (the residual mass is at rounding level or zero):
         // go over the whole row in double precision.
@@ -1032,6 +1038,7 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
         block_argmax(score, Z, s_score, s_x);
         if (!(score > -INFINITY)) {
             // [pi - rho]_+ is identically zero: commit arg-max of pi (= arg-max of the target logits)
+            have_score = false;
             score = -INFINITY;
             Z = 0x7FFFFFFF;
             for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
@@ -1045,10 +1052,191 @@ __global__ void __launch_bounds__(kResidualThreads, 4) residual_kernel(const __g
         }
     }
     if (threadIdx.x == 0) {
-        const double lp = load_logit<DT>(prow, Z);
-        P.tokens[row] = Z;
-        P.conf[row] = static_cast<float>(exp2(lp * c - task.kp));
+        // Z stays "none" when the row (vocabulary-parallel mode: this rank's slice of it) holds no finite
+        // target logit; a whole row like that has been reported by the scan already
+        const bool none = Z < 0 || Z >= G.V;
+        const float lp = none ? -INFINITY : load_logit<DT>(prow, Z);
+        if (none && !P.vp_out) {
+            P.tokens[row] = -1;
+            P.conf[row] = -1.f;
+            report(P.status, FEF_ERR_NONFINITE);
+        } else if (P.vp_out) {  // vocabulary-parallel: this rank's best; the ranks' reports are compared afterwards
+            VpCandidate out;
+            out.score = (have_score && !none) ? score : -INFINITY;
+            out.lp = lp;
+            out.index = none ? 0x7FFFFFFF : Z + P.vocab_offset;
+            P.vp_out[b] = out;
+        } else {
+            P.tokens[row] = Z;
+            P.conf[row] = static_cast<float>(exp2(static_cast<double>(lp) * c - task.kp));
+        }
     }
+}
+
+// =================================================== vocabulary-parallel ====
+// The same verification when the vocabulary axis is split over ranks (logits leaving a
+// tensor-parallel LM head): every rank streams its slice once, the ranks exchange six numbers
+// per position, decide the acceptance tests identically, draw their share of each residual
+// sample over their slice and exchange one candidate per rejected window.
+constexpr int kVpStatsPerRow = 6;  // M_p, S_p, M_q, S_q, l^p[x], l^q[x]
+
+// Per row of this rank's slice: the (reference, sum) pairs of the two laws and, on the rank whose
+// slice holds the draft token, the two logits at it (NaN elsewhere).  S = NaN marks bad data.
+template <int DT>
+__global__ void __launch_bounds__(128) vp_stats_kernel(const __grid_constant__ VerifyParams P, double* __restrict__ stats) {
+    const Geometry& G = P.geo;
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (row >= static_cast<int64_t>(G.B) * G.K) return;
+    const int b = static_cast<int>(row / G.K), i = static_cast<int>(row - static_cast<int64_t>(b) * G.K);
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    const double nan = __longlong_as_double(0x7FF8000000000000ll);
+    double out[kVpStatsPerRow] = {-INFINITY, 0.0, -INFINITY, 0.0, nan, nan};
+    if (i < n) {
+        const char* prow = P.target + row * G.ld_bytes;
+        const char* qrow = P.draft + row * G.ld_bytes;
+        const RowNorm np = fold_unit<DT, false>(2 * row, prow, c, P);
+        const RowNorm nq = fold_unit<DT, false>(2 * row + 1, qrow, c, P);
+        out[0] = np.M;
+        out[1] = np.data_bad ? nan : np.S;
+        out[2] = nq.M;
+        out[3] = nq.data_bad ? nan : nq.S;
+        const int x = __ldg(P.draft_tokens + row) - P.vocab_offset;
+        if (x >= 0 && x < G.V) {
+            out[4] = load_logit<DT>(prow, x);
+            out[5] = load_logit<DT>(qrow, x);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kVpStatsPerRow; ++k) stats[row * kVpStatsPerRow + k] = out[k];
+}
+
+// The ranks' (reference, sum) pairs of one law folded into its log2 normaliser; false on bad data.
+__device__ bool vp_fold(const double* __restrict__ stats, int ranks, int64_t rows, int64_t row, int at, double* k_out) {
+    double M = -INFINITY, S = 0.0;
+    bool bad = false;
+    for (int r = 0; r < ranks; ++r) {
+        const double* rec = stats + (static_cast<int64_t>(r) * rows + row) * kVpStatsPerRow + at;
+        const double m = rec[0], sum = rec[1];
+        if (!(sum >= 0.0) || sum == INFINITY) bad = true;
+        if (sum > 0.0) {
+            if (m > M) {
+                S = S * exp2(M - m) + sum;
+                M = m;
+            } else {
+                S += sum * exp2(m - M);
+            }
+        }
+    }
+    if (bad || !(S > 0.0) || !(S < INFINITY)) return false;
+    *k_out = M + log2(S);
+    return true;
+}
+
+// Acceptance tests, first rejection and outputs from the gathered statistics: one CTA per
+// window, one thread per position; every rank runs it on the same numbers.
+__global__ void __launch_bounds__(FEF_MAX_K) vp_accept_kernel(const __grid_constant__ VerifyParams P,
+                                                              const double* __restrict__ stats, int ranks, int V_total) {
+    const Geometry& G = P.geo;
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    const int64_t rows = static_cast<int64_t>(G.B) * G.K, row = static_cast<int64_t>(b) * G.K + i;
+    __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K];
+    __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
+    int tok = -1;
+    float conf = -1.f;
+    if (i < n) {
+        int err = 0, accept = 0;
+        double kp = 0.0, kq = 0.0;
+        tok = __ldg(P.draft_tokens + row);
+        double lpx = 0.0, lqx = 0.0;
+        int owners = 0;
+        for (int r = 0; r < ranks; ++r) {
+            const double* rec = stats + (static_cast<int64_t>(r) * rows + row) * kVpStatsPerRow;
+            if (rec[4] == rec[4]) {  // not NaN: this rank holds the token
+                lpx = rec[4];
+                lqx = rec[5];
+                ++owners;
+            }
+        }
+        if (tok < 0 || tok >= V_total || owners != 1) {
+            err = FEF_ERR_TOKEN_RANGE;
+        } else if (!vp_fold(stats, ranks, rows, row, 0, &kp) || !vp_fold(stats, ranks, rows, row, 2, &kq)) {
+            err = FEF_ERR_NONFINITE;
+        } else {
+            const double l2pi = lpx * c - kp;  // log2 pi(x)
+            conf = static_cast<float>(exp2(l2pi));
+            if (lqx == -INFINITY) {
+                accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
+            } else {
+                const double ratio = exp2(l2pi - (lqx * c - kq));
+                const uint4 r = philox4x32_10(
+                    make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
+                    make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+                accept = static_cast<double>(uniform_from_word(r.x)) <= fmin(1.0, ratio);
+            }
+        }
+        s_err[i] = err;
+        s_accept[i] = accept;
+        s_kp[i] = kp;
+        s_kq[i] = kq;
+    }
+    __syncthreads();
+    int err = 0, a = n;
+    for (int k = 0; k < n; ++k) err = max(err, s_err[k]);
+    for (int k = n - 1; k >= 0; --k)
+        if (!s_accept[k]) a = k;
+    if (i < G.K) {
+        const bool keep = !err && i < a;
+        P.tokens[row] = keep ? tok : -1;
+        P.conf[row] = keep ? conf : -1.f;
+    }
+    if (i == 0) {
+        P.accept_len[b] = err ? -1 : a;
+        if (err) report(P.status, err);
+        ResidualTask task;
+        task.pos = (!err && a < n) ? a : -1;
+        task.arrivals = 0u;
+        task.kp = task.pos >= 0 ? s_kp[a] : 0.0;
+        task.kq = task.pos >= 0 ? s_kq[a] : 0.0;
+        P.tasks[b] = task;
+    }
+}
+
+// The ranks' candidates of each rejected window compared: the largest exact score wins (lowest
+// id on ties); if no rank has a positive residual weight, the largest target logit does.
+__global__ void __launch_bounds__(128) vp_finish_kernel(const __grid_constant__ VerifyParams P,
+                                                        const VpCandidate* __restrict__ cands, int ranks) {
+    const Geometry& G = P.geo;
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= G.B) return;
+    const ResidualTask task = P.tasks[b];
+    if (task.pos < 0) return;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    double best = -INFINITY;
+    float best_lp = -INFINITY, lp = 0.f;
+    int Z = 0x7FFFFFFF, Zl = 0x7FFFFFFF;
+    for (int r = 0; r < ranks; ++r) {
+        const VpCandidate cd = cands[static_cast<int64_t>(r) * G.B + b];
+        if (cd.score > best || (cd.score == best && cd.score > -INFINITY && cd.index < Z)) {
+            best = cd.score;
+            Z = cd.index;
+            lp = cd.lp;
+        }
+        if (cd.lp > best_lp || (cd.lp == best_lp && cd.index < Zl)) {
+            best_lp = cd.lp;
+            Zl = cd.index;
+        }
+    }
+    if (!(best > -INFINITY)) {  // [pi - rho]_+ is zero everywhere: arg-max of pi
+        Z = Zl;
+        lp = best_lp;
+    }
+    const int64_t row = static_cast<int64_t>(b) * G.K + task.pos;
+    P.tokens[row] = Z;
+    P.conf[row] = static_cast<float>(exp2(static_cast<double>(lp) * c - task.kp));
 }
 
 // ================================================================= host ====
@@ -1303,6 +1491,8 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
     P.partials = reinterpret_cast<Partial*>(ws + L.partials);
     P.tasks = reinterpret_cast<ResidualTask*>(ws + L.tasks);
     P.candidates = reinterpret_cast<Candidate*>(ws + L.candidates);
+    P.vocab_offset = 0;
+    P.vp_out = nullptr;
     P.status = device_status;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -1362,6 +1552,165 @@ fef_status fef_spec_verify_at_round(const void* draft_logits, const void* target
     return verify_impl(draft_logits, target_logits, draft_tokens, row_len, draft_log2_norm, B, K, V, ld, dt,
                        temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes, device_status,
                        cuda_stream, nullptr, device_round);
+}
+
+}  // extern "C"
+
+// Parameter block of a vocabulary-parallel call on this rank's slice (no launch).
+static fef_status vp_setup(const void* draft_slice, const void* target_slice, const int32_t* draft_tokens,
+                           const int32_t* row_len, int B, int K, int V_local, int64_t ld, fef_dtype dt,
+                           float temperature, uint64_t seed, uint32_t step, int vocab_offset, void* workspace,
+                           size_t workspace_bytes, bool need_logits, fef::VerifyParams* out, int* dev_out) {
+    using namespace fef;
+    if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
+    if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V_local < 1 || ld < V_local) return FEF_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || isinf(temperature)) return FEF_ERR_INVALID_ARG;  // sampling mode only
+    if (vocab_offset < 0 || (vocab_offset & 7)) return FEF_ERR_INVALID_ARG;
+    const int esize = dt == FEF_F32 ? 4 : 2;
+    if (static_cast<int64_t>(V_local) * esize > (1ll << 30)) return FEF_ERR_INVALID_ARG;
+    if (need_logits) {
+        if (!draft_slice || !target_slice) return FEF_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(draft_slice) & 15) || (reinterpret_cast<uintptr_t>(target_slice) & 15) ||
+            ((ld * esize) & 15))
+            return FEF_ERR_ALIGNMENT;
+    }
+    const int sms = sm_count_of_current_device(dev_out);
+    if (sms < 1) return FEF_ERR_CUDA;
+    VerifyParams P = {};
+    if (!make_geometry(B, K, V_local, ld, dt, false, sms, &P.geo)) return FEF_ERR_INVALID_ARG;
+    const double c = 1.4426950408889634074 / static_cast<double>(temperature);
+    float c_hi = static_cast<float>(c);
+    if (dt == FEF_F32) {
+        if (static_cast<double>(c_hi) >= c) c_hi = nextafterf(c_hi, 0.0f);
+        P.c_lo = static_cast<float>(c - static_cast<double>(c_hi));
+        if (!(P.c_lo > 0.f)) return FEF_ERR_INVALID_ARG;
+    }
+    P.c_hi = c_hi;
+    if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
+    P.target = static_cast<const char*>(target_slice);
+    P.draft = static_cast<const char*>(draft_slice);
+    P.draft_tokens = draft_tokens;
+    P.row_len = row_len;
+    P.seed = seed;
+    P.keys = philox_round_keys(seed);
+    P.step = step;
+    P.vocab_offset = vocab_offset;
+    if (workspace) {
+        const WorkspaceLayout L = layout_of(P.geo);
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total) return FEF_ERR_WORKSPACE;
+        char* ws = static_cast<char*>(workspace);
+        P.ctl = reinterpret_cast<Control*>(ws + L.control);
+        P.partials = reinterpret_cast<Partial*>(ws + L.partials);
+        P.candidates = reinterpret_cast<Candidate*>(ws + L.candidates);
+    }
+    *out = P;
+    return FEF_OK;
+}
+
+template <int DT>
+static cudaError_t vp_launch_stats(const fef::VerifyParams& P, int dev, double* stats, cudaStream_t stream) {
+    using namespace fef;
+    const Geometry& G = P.geo;
+    const int which = DT * 2;
+    if (!g_attr_done[dev][which]) {
+        const cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(kSmemBytes));
+        if (e != cudaSuccess) return e;
+        g_attr_done[dev][which] = true;
+    }
+    cudaError_t e = launch_dependent(begin_call_kernel, dim3(1), dim3(32), 0, stream, P.ctl, P.status);
+    if (e != cudaSuccess) return e;
+    e = launch_dependent(stream_kernel<DT, false>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
+    if (e != cudaSuccess) return e;
+    const int64_t rows = static_cast<int64_t>(G.B) * G.K;
+    return launch_dependent(vp_stats_kernel<DT>, dim3(static_cast<unsigned>((rows + 127) / 128)), dim3(128), 0, stream, P,
+                            stats);
+}
+
+extern "C" {
+
+size_t fef_vp_task_bytes(int B) { return B < 1 ? 0 : static_cast<size_t>(B) * sizeof(fef::ResidualTask); }
+
+fef_status fef_vp_local_stats(const void* draft_slice, const void* target_slice, const int32_t* draft_tokens,
+                              const int32_t* row_len, int B, int K, int V_local, int64_t ld, fef_dtype dt,
+                              float temperature, int vocab_offset, double* stats, void* workspace,
+                              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    using namespace fef;
+    if (!draft_tokens || !stats || !workspace) return FEF_ERR_INVALID_ARG;
+    VerifyParams P;
+    int dev = 0;
+    const fef_status st = vp_setup(draft_slice, target_slice, draft_tokens, row_len, B, K, V_local, ld, dt, temperature,
+                                   0, 0, vocab_offset, workspace, workspace_bytes, true, &P, &dev);
+    if (st != FEF_OK) return st;
+    P.status = device_status;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t e = dt == FEF_F32 ? vp_launch_stats<FEF_F32>(P, dev, stats, stream)
+                                        : vp_launch_stats<FEF_BF16>(P, dev, stats, stream);
+    return e == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_vp_accept(const double* stats_all, int ranks, const int32_t* draft_tokens, const int32_t* row_len,
+                         int B, int K, int V_total, fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
+                         int32_t* accept_len, int32_t* tokens, float* conf, void* tasks, int32_t* device_status,
+                         void* cuda_stream) {
+    using namespace fef;
+    if (!stats_all || ranks < 1 || ranks > 1024 || !draft_tokens || !accept_len || !tokens || !conf || !tasks ||
+        V_total < 1)
+        return FEF_ERR_INVALID_ARG;
+    VerifyParams P;
+    int dev = 0;
+    // (the slice width only shapes the streaming geometry, which this step does not use)
+    const fef_status st = vp_setup(nullptr, nullptr, draft_tokens, row_len, B, K, 8, 8, dt, temperature, seed, step, 0,
+                                   nullptr, 0, false, &P, &dev);
+    if (st != FEF_OK) return st;
+    P.accept_len = accept_len;
+    P.tokens = tokens;
+    P.conf = conf;
+    P.tasks = static_cast<ResidualTask*>(tasks);
+    P.status = device_status;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (device_status && cudaMemsetAsync(device_status, 0, sizeof(int32_t), stream) != cudaSuccess) return FEF_ERR_CUDA;
+    vp_accept_kernel<<<B, FEF_MAX_K, 0, stream>>>(P, stats_all, ranks, V_total);
+    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_vp_local_residual(const void* draft_slice, const void* target_slice, void* tasks, int B, int K,
+                                 int V_local, int64_t ld, fef_dtype dt, float temperature, uint64_t seed,
+                                 uint32_t step, int vocab_offset, void* candidates, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    using namespace fef;
+    if (!tasks || !candidates || !workspace) return FEF_ERR_INVALID_ARG;
+    VerifyParams P;
+    int dev = 0;
+    const fef_status st = vp_setup(draft_slice, target_slice, nullptr, nullptr, B, K, V_local, ld, dt, temperature, seed,
+                                   step, vocab_offset, workspace, workspace_bytes, true, &P, &dev);
+    if (st != FEF_OK) return st;
+    P.tasks = static_cast<ResidualTask*>(tasks);
+    P.vp_out = static_cast<VpCandidate*>(candidates);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const dim3 grid(P.geo.residual_ctas, B);
+    if (dt == FEF_F32)
+        residual_kernel<FEF_F32><<<grid, kResidualThreads, 0, stream>>>(P);
+    else
+        residual_kernel<FEF_BF16><<<grid, kResidualThreads, 0, stream>>>(P);
+    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+}
+
+fef_status fef_vp_finish(const void* candidates_all, int ranks, const void* tasks, int B, int K, fef_dtype dt,
+                         float temperature, int32_t* tokens, float* conf, void* cuda_stream) {
+    using namespace fef;
+    if (!candidates_all || ranks < 1 || ranks > 1024 || !tasks || !tokens || !conf) return FEF_ERR_INVALID_ARG;
+    VerifyParams P;
+    int dev = 0;
+    const fef_status st = vp_setup(nullptr, nullptr, nullptr, nullptr, B, K, 8, 8, dt, temperature, 0, 0, 0, nullptr, 0,
+                                   false, &P, &dev);
+    if (st != FEF_OK) return st;
+    P.tokens = tokens;
+    P.conf = conf;
+    P.tasks = static_cast<ResidualTask*>(const_cast<void*>(tasks));
+    vp_finish_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        P, static_cast<const VpCandidate*>(candidates_all), ranks);
+    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 // ---- host-buffer variant: layout of the caller's device arena

@@ -138,6 +138,22 @@ a = oracle.spec_verify(q, p, tok, 1.0, du.rank_seed(7, rank), 3)["tokens"]
 gathered = [torch.zeros((w.B, w.K), dtype=torch.int32) for _ in range(world)]
 dist.all_gather(gathered, torch.as_tensor(a))
 assert any((gathered[0] != g).any() for g in gathered[1:])
+# vocabulary-parallel exchange: every rank reduces its slice to (reference, sum) per row; gathered
+# rank-major (the layout fef_vp_accept reads) and folded, they give the full rows' normalisers
+from paper_2605_14305_b200.vocab_parallel import shard_vocab, STATS_PER_ROW
+rows = q.reshape(-1, w.V).double()
+off, width = shard_vocab(w.V, world)[rank]
+sl = rows[:, off:off + width]
+mine = torch.zeros((rows.shape[0], STATS_PER_ROW), dtype=torch.float64)
+mine[:, 0] = sl.max(dim=1).values
+mine[:, 1] = torch.exp2(sl - mine[:, :1]).sum(dim=1)
+everyone = torch.empty((world * mine.shape[0], STATS_PER_ROW), dtype=torch.float64)
+dist.all_gather_into_tensor(everyone, mine)
+everyone = everyone.reshape(world, mine.shape[0], STATS_PER_ROW)
+M = everyone[:, :, 0].max(dim=0).values
+S = (everyone[:, :, 1] * torch.exp2(everyone[:, :, 0] - M)).sum(dim=0)
+assert torch.allclose(M + torch.log2(S), torch.log2(torch.exp2(rows).sum(dim=1)), rtol=1e-12, atol=1e-12)
+assert off %% 8 == 0 and sum(wd for _, wd in shard_vocab(w.V, world)) == w.V
 rate = du.aggregate_rate(w.B * w.K, 4, got[0], world)
 if rank == 0:
     print(json.dumps({"ok": True, "rate": rate}))

@@ -36,6 +36,7 @@ struct Geometry {
     int tiles_per_claim;  // tiles one claim covers
     int claims_per_unit;  // claims per row (>= 1, also for rows without a whole vector)
     int grid;             // CTAs of the streaming kernel
+    int warp_per_row;     // 1: short rows, many of them: rows_kernel (one warp per row) streams instead
     int residual_ctas;    // CTAs per rejected row in the residual kernel
     int64_t num_units;    // rows to stream: B * K * units_per_row
     int64_t num_claims;   // num_units * claims_per_unit
@@ -421,6 +422,72 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             for (int spin = 0; spin < kSpinLimit; ++spin)
                 if (mbar_try_wait(full + s, phase)) break;
         }
+    }
+}
+
+// ========================================================= short rows ====
+// The same sums for rows that fit one tile when there are many of them (small vocabularies,
+// slices of a sharded vocabulary): one warp per row and tensor, four 16-byte loads per lane in
+// flight, one warp reduction per row, no shared memory.  Leaves one partial per row like the ring.
+constexpr int kRowsWarps = 8;        // rows a CTA works on at a time
+constexpr int kRowsCtasPerSm = 4;
+
+template <int DT, bool GREEDY>
+__global__ void __launch_bounds__(kRowsWarps * 32, kRowsCtasPerSm) rows_kernel(const __grid_constant__ VerifyParams P) {
+    const Geometry& G = P.geo;
+    cudaGridDependencySynchronize();  // an earlier call on the stream may still be reading the partials
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kRowsWarps;
+    for (int64_t unit = static_cast<int64_t>(blockIdx.x) * kRowsWarps + warp; unit < G.num_units; unit += stride) {
+        const int64_t row = G.units_per_row == 2 ? (unit >> 1) : unit;
+        const bool is_draft = G.units_per_row == 2 && (unit & 1);
+        const int b = static_cast<int>(row / G.K), i = static_cast<int>(row - static_cast<int64_t>(b) * G.K);
+        const int n = P.row_len ? __ldg(P.row_len + b) : G.K;
+        RowState st;
+        st.reset();
+        if (i < n) {
+            const char* base = (is_draft ? P.draft : P.target) + row * G.ld_bytes;
+            const int len = G.vec_bytes;
+            // two batches of four vectors per lane are in flight: the second is issued before the first
+            // is added up
+            constexpr int kBatchBytes = 32 * 16 * kVecPerThread;
+            // (the loop bounds are the same in every lane: the warp votes of greedy mode need the whole warp)
+            for (int off = 0; off < len; off += 2 * kBatchBytes) {
+                uint4 w[2][kVecPerThread];
+                int at[2][kVecPerThread];
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        at[h][j] = off + h * kBatchBytes + j * 32 * 16 + lane * 16;
+                        if (at[h][j] < len) w[h][j] = ld_global_nc_v4(base + at[h][j]);
+                    }
+                if (st.ref == kNoReference && at[0][0] < len) st.ref = first_reference<DT>(w[0][0], P.c_hi, P.c_lo);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (off + h * kBatchBytes >= len) break;  // uniform over the warp
+                    float tile_sum;
+                    if (at[h][kVecPerThread - 1] < len)
+                        tile_sum = absorb_tile<DT, true>(w[h], at[h], len, P.c_hi, P.c_lo, st);
+                    else
+                        tile_sum = absorb_tile<DT, false>(w[h], at[h], len, P.c_hi, P.c_lo, st);
+                    if constexpr (GREEDY) {
+                        const float floor_f = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(st.best)));
+                        // 0.999: the sum and the bound carry a few units of 1e-7 of rounding each
+                        const bool candidate = !(tile_sum < 0.999f * exp2_scaled<DT>(floor_f, P.c_hi, P.c_lo, st.ref));
+                        if (__any_sync(0xFFFFFFFFu, candidate)) {
+                            if (candidate) {
+#pragma unroll
+                                for (int j = 0; j < kVecPerThread; ++j)
+                                    if (at[h][j] < len) track_best<DT>(w[h][j], at[h][j] / Elem<DT>::kBytes, st);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        const Partial all = warp_combine<GREEDY>(st.ref, st.sum, st.best, st.index);
+        if (lane == 0) P.partials[unit] = all;
     }
 }
 
@@ -1296,6 +1363,17 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool ta
     G.num_claims = G.num_units * G.claims_per_unit;
     if (G.num_claims >= (1ll << 31)) return false;  // claim numbers are handled as 32-bit values
     G.grid = static_cast<int>(G.num_claims < sm_count ? G.num_claims : sm_count);
+    // Rows of at most one tile, enough of them to give every resident warp its own: the ring would
+    // end every tile in a cross-warp combine, so a warp takes a whole row instead
+    G.warp_per_row = (G.vec_bytes > 0 && G.vec_bytes <= kTileBytes &&
+                      G.num_units >= static_cast<int64_t>(sm_count) * kRowsWarps * 2) ? 1 : 0;
+    if (G.warp_per_row) {
+        G.claims_per_unit = 1;
+        G.num_claims = G.num_units;
+        const int64_t ctas = (G.num_units + kRowsWarps - 1) / kRowsWarps;
+        const int64_t cap = static_cast<int64_t>(sm_count) * kRowsCtasPerSm;
+        G.grid = static_cast<int>(ctas < cap ? ctas : cap);
+    }
 
     // residual kernel: CTAs per rejected row, each thread up to kResidualBatch vector pairs
     // (fewer when few windows would leave SMs idle)
@@ -1368,7 +1446,12 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         g_attr_done[dev][which] = true;
     }
     cudaError_t e;
-    if (events) {
+    if (G.warp_per_row) {
+        if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
+        mark(events, 0, stream);
+        e = launch_dependent(rows_kernel<DT, GREEDY>, dim3(G.grid), dim3(kRowsWarps * 32), 0, stream, P);
+        if (e != cudaSuccess) return e;
+    } else if (events) {
         // timing marks asked for: clear with memset nodes and launch the streaming kernel the
         // ordinary way, so that the first two marks bracket that kernel alone
         if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
@@ -1618,9 +1701,15 @@ static cudaError_t vp_launch_stats(const fef::VerifyParams& P, int dev, double* 
         if (e != cudaSuccess) return e;
         g_attr_done[dev][which] = true;
     }
-    cudaError_t e = launch_dependent(begin_call_kernel, dim3(1), dim3(32), 0, stream, P.ctl, P.status);
-    if (e != cudaSuccess) return e;
-    e = launch_dependent(stream_kernel<DT, false>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
+    cudaError_t e;
+    if (G.warp_per_row) {
+        if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
+        e = launch_dependent(rows_kernel<DT, false>, dim3(G.grid), dim3(kRowsWarps * 32), 0, stream, P);
+    } else {
+        e = launch_dependent(begin_call_kernel, dim3(1), dim3(32), 0, stream, P.ctl, P.status);
+        if (e != cudaSuccess) return e;
+        e = launch_dependent(stream_kernel<DT, false>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
+    }
     if (e != cudaSuccess) return e;
     const int64_t rows = static_cast<int64_t>(G.B) * G.K;
     return launch_dependent(vp_stats_kernel<DT>, dim3(static_cast<unsigned>((rows + 127) / 128)), dim3(128), 0, stream, P,

@@ -56,6 +56,8 @@ SMALL_SHAPES = [
     (1, 1, 1, 4), (2, 3, 3, 4), (3, 2, 4, 4), (2, 4, 7, 8), (5, 4, 8, 8), (2, 5, 9, 12), (3, 7, 33, 36),
     (4, 4, 1000, 1000), (1, 4, 1024, 1024), (2, 3, 4097, 4104), (7, 32, 260, 264), (2, 64, 520, 520),
     (300, 2, 64, 64), (2, 2, 40000, 40000), (1, 3, 70001, 70008),
+    # short rows, many of them: the warp-per-row streaming kernel
+    (40, 32, 1000, 1000), (100, 16, 4097, 4104), (1300, 1, 24, 24), (64, 32, 15808, 15808),
 ]
 
 

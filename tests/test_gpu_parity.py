@@ -444,6 +444,7 @@ def test_draft_tokens_feed_verification(fef):
 def test_verification_with_the_draft_normalisers_streams_the_target_only(fef):
     """fef_draft_sample -> fef_spec_verify_with_draft_norm against the oracle pair, and against the plain call."""
     for w, T, seed in ((synth.LLADA_BATCHED.with_(B=5, K=16), 0.7, 41), (synth.LLADA_SINGLE.with_(K=8), 1.0, 42),
+                       (synth.TINY.with_(B=90, K=32, V=3000, dtype=torch.bfloat16), 1.0, 44),  # short rows: warp per row
                        (synth.DREAM_LARGE.with_(B=3, K=8, dtype=torch.float32), 1.0, 43)):
         q, p = synth.make_logits(w, seed=seed, device="cuda")
         d = fef.fef_draft_sample(q, T, seed, 7)

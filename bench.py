@@ -434,6 +434,43 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------- loop sweep ----
+def run_loop_sweep(args):
+    """Extra mode (not the contract's line): the long-generation sweep — the full decoding loop
+    (window, draft draws, verification, commit; re-masking between two denoising steps) on a
+    device-resident state of L = 1024 positions per sequence until nothing is masked, at
+    B in {1, 8, 64} x K in {8, 32, 64}, bf16 and fp32, eager and as a replayed CUDA graph.
+    The logits are fixed tensors made before the loop (their generation is not in the time)."""
+    import paper_2605_14305_b200 as fef
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device, run_decode_loop_graph
+
+    fef.load(build_if_missing=True)
+    torch.cuda.set_device(0)
+    L, remask_k = 1024, 8
+    points = []
+    for dtype in (torch.bfloat16, torch.float32):
+        for B in (1, 8, 64):
+            for K in (8, 32, 64):
+                w = synth.HEADLINE.with_(B=B, K=K, dtype=dtype, noise_std=0.7)
+                t0 = time.perf_counter()
+                q, p = synth.make_logits(w, seed=args.seed, device="cuda")
+                torch.cuda.synchronize()
+                gen_s = time.perf_counter() - t0
+                res = {}
+                for name, fn, lf in (("eager", run_decode_loop_device, lambda rnd, window, row_len, inputs: (q, p)),
+                                     ("graph", run_decode_loop_graph, lambda rnd, window, row_len: (q, p))):
+                    fn(fef, B, L, K, 2, remask_k, lf, w.temperature, args.seed)       # warm-up
+                    out = fn(fef, B, L, K, 2, remask_k, lf, w.temperature, args.seed)
+                    res[name] = {"rounds": out["rounds"], "us_per_round": out["loop_seconds"] * 1e6 / out["rounds"],
+                                 "committed_positions_per_s": (B * L + B * remask_k) / out["loop_seconds"]}
+                points.append({"B": B, "K": K, "dtype": "bf16" if dtype == torch.bfloat16 else "f32",
+                               "logit_generation_s": gen_s, **res})
+                del q, p
+    print(json.dumps({"mode": "loop sweep", "L": L, "V": synth.HEADLINE.V, "denoising_steps": 2, "remask_k": remask_k,
+                      "verification": "fef_draft_sample + fef_spec_verify reusing the draft normalisers",
+                      "data": "synthetic", "points": points}))
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--gpus", type=int, default=1)
@@ -453,8 +490,11 @@ def main():
     ap.add_argument("--cpu-windows", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-call-events", action="store_true")
+    ap.add_argument("--loop-sweep", action="store_true", help="time the full decoding loop at the sweep points instead")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.loop_sweep:
+        run_loop_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_native(args)

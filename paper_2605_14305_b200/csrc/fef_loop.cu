@@ -18,6 +18,7 @@ __global__ void __launch_bounds__(kLoopThreads) next_window_kernel(const int32_t
                                                                    int32_t* __restrict__ window_pos,
                                                                    int32_t* __restrict__ row_len,
                                                                    int32_t* __restrict__ unresolved) {
+    cudaGridDependencySynchronize();  // launched while its predecessor on the stream drains
     __shared__ int s_warp[kLoopThreads / 32];
     const int b = blockIdx.x;
     const int32_t* row = tokens + static_cast<int64_t>(b) * L;
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(kLoopThreads) inputs_kernel(const int32_t* __r
                                                               const int32_t* __restrict__ row_len,
                                                               const int32_t* __restrict__ draft_tokens, int L, int K,
                                                               int32_t* __restrict__ inputs) {
+    cudaGridDependencySynchronize();  // launched while its predecessor on the stream drains
     const int b = blockIdx.x / K, m = blockIdx.x - b * K;
     const int32_t* row = tokens + static_cast<int64_t>(b) * L;
     int32_t* out = inputs + static_cast<int64_t>(blockIdx.x) * L;
@@ -75,6 +77,7 @@ __global__ void commit_kernel(const int32_t* __restrict__ window_pos, const int3
                               const float* __restrict__ out_conf, int B, int L, int K, int32_t* __restrict__ tokens,
                               float* __restrict__ conf, uint8_t* __restrict__ in_step,
                               int32_t* __restrict__ committed) {
+    cudaGridDependencySynchronize();  // launched while its predecessor on the stream drains
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= B * K) return;
     const int b = idx / K, t = idx - b * K;
@@ -94,6 +97,7 @@ __global__ void commit_kernel(const int32_t* __restrict__ window_pos, const int3
 __global__ void remask_apply_kernel(const int32_t* __restrict__ positions, const int32_t* __restrict__ count, int L,
                                     int k, int32_t* __restrict__ tokens, float* __restrict__ conf,
                                     uint8_t* __restrict__ in_step) {
+    cudaGridDependencySynchronize();  // launched while its predecessor on the stream drains
     const int b = blockIdx.x;
     for (int j = threadIdx.x; j < L; j += blockDim.x) in_step[static_cast<int64_t>(b) * L + j] = 0;
     const int n = min(count[b], k);
@@ -110,11 +114,28 @@ __global__ void remask_apply_kernel(const int32_t* __restrict__ positions, const
 // unless `unresolved` is given and no row has an unresolved position left (a replayed round
 // that had nothing to do takes no number).
 __global__ void __launch_bounds__(kLoopThreads) advance_round_kernel(uint32_t* round, const int32_t* unresolved, int B) {
+    cudaGridDependencySynchronize();  // launched while its predecessor on the stream drains
     int any = unresolved ? 0 : 1;
     if (unresolved)
         for (int b = threadIdx.x; b < B; b += kLoopThreads) any |= unresolved[b] > 0;
     any = __syncthreads_or(any);
     if (threadIdx.x == 0 && any) *round += 1u;
+}
+
+// Programmatic dependent launch: the grid may be scheduled while its predecessor on the stream
+// drains; every kernel here waits (cudaGridDependencySynchronize) before it touches memory.
+template <typename... Args>
+static cudaError_t launch_chained(void (*kernel)(Args...), dim3 grid, dim3 block, void* cuda_stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 static bool loop_sizes_ok(int B, int L, int K) {
@@ -129,9 +150,7 @@ fef_status fef_loop_next_window(const int32_t* tokens, int B, int L, int K, int3
                                 int32_t* unresolved, void* cuda_stream) {
     using namespace fef;
     if (!tokens || !window_pos || !row_len || !unresolved || !loop_sizes_ok(B, L, K)) return FEF_ERR_INVALID_ARG;
-    next_window_kernel<<<B, kLoopThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(tokens, L, K, window_pos, row_len,
-                                                                                      unresolved);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    return fef::launch_chained(fef::next_window_kernel, dim3(B), dim3(kLoopThreads), cuda_stream, tokens, L, K, window_pos, row_len, unresolved) == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 fef_status fef_loop_verification_inputs(const int32_t* tokens, const int32_t* window_pos, const int32_t* row_len,
@@ -140,9 +159,7 @@ fef_status fef_loop_verification_inputs(const int32_t* tokens, const int32_t* wi
     using namespace fef;
     if (!tokens || !window_pos || !row_len || !draft_tokens || !inputs || !loop_sizes_ok(B, L, K))
         return FEF_ERR_INVALID_ARG;
-    inputs_kernel<<<B * K, kLoopThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(tokens, window_pos, row_len,
-                                                                                     draft_tokens, L, K, inputs);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    return fef::launch_chained(fef::inputs_kernel, dim3(B * K), dim3(kLoopThreads), cuda_stream, tokens, window_pos, row_len, draft_tokens, L, K, inputs) == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 fef_status fef_loop_commit(const int32_t* window_pos, const int32_t* row_len, const int32_t* accept_len,
@@ -153,9 +170,7 @@ fef_status fef_loop_commit(const int32_t* window_pos, const int32_t* row_len, co
         !committed || !loop_sizes_ok(B, L, K))
         return FEF_ERR_INVALID_ARG;
     const int threads = 256, blocks = (B * K + threads - 1) / threads;
-    commit_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        window_pos, row_len, accept_len, out_tokens, out_conf, B, L, K, tokens, conf, in_step, committed);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    return fef::launch_chained(fef::commit_kernel, dim3(blocks), dim3(threads), cuda_stream, window_pos, row_len, accept_len, out_tokens, out_conf, B, L, K, tokens, conf, in_step, committed) == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B, int L, int k, int32_t* tokens,
@@ -163,16 +178,12 @@ fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B
     using namespace fef;
     if (!count || !tokens || !conf || !in_step || k < 0 || (k > 0 && !positions) || !loop_sizes_ok(B, L, 1))
         return FEF_ERR_INVALID_ARG;
-    remask_apply_kernel<<<B, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(positions, count, L, k, tokens, conf,
-                                                                              in_step);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    return fef::launch_chained(fef::remask_apply_kernel, dim3(B), dim3(256), cuda_stream, positions, count, L, k, tokens, conf, in_step) == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 fef_status fef_loop_advance_round(uint32_t* device_round, const int32_t* unresolved, int B, void* cuda_stream) {
     if (!device_round || (unresolved && (B < 1 || B > FEF_MAX_B))) return FEF_ERR_INVALID_ARG;
-    fef::advance_round_kernel<<<1, fef::kLoopThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(device_round,
-                                                                                                 unresolved, B);
-    return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
+    return fef::launch_chained(fef::advance_round_kernel, dim3(1), dim3(fef::kLoopThreads), cuda_stream, device_round, unresolved, B) == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -1310,7 +1310,7 @@ __global__ void __launch_bounds__(128) vp_finish_kernel(const __grid_constant__ 
 static int g_sm_count[64];
 static bool g_attr_done[64][4];
 
-constexpr int kClaimsPerCta = 6;             // streaming claims a CTA should get at least, size permitting
+constexpr int kClaimsPerCta = 3;             // streaming claims a CTA should get at least, size permitting (6 cost B = 1 calls 4 us)
 constexpr int kMaxClaimBytes = 1 << 20;      // and at most this many bytes per claim (a whole row of the usual sizes)
 
 static int sm_count_of_current_device(int* device_out) {

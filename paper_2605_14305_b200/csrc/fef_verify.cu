@@ -789,18 +789,42 @@ constexpr int kScanMaxWarps = 32;
 template <int DT, bool GREEDY>
 __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __grid_constant__ VerifyParams P) {
     const Geometry& G = P.geo;
-    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
     const int num_warps = blockDim.x >> 5;
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
     const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
 
+    // what does not depend on the streaming kernel is fetched before waiting for it: the draft
+    // tokens of this warp's positions and the logits at them (a warp has at most kRows positions)
+    constexpr int kRows = (FEF_MAX_K + kScanMaxWarps - 1) / kScanMaxWarps;
+    int pre_x[kRows];
+    double pre_lp[kRows], pre_lq[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        const int i = warp + r * num_warps;
+        pre_x[r] = -1;
+        pre_lp[r] = pre_lq[r] = 0.0;
+        if (lane == 0 && i < n) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
+            const int x = __ldg(P.draft_tokens + row);
+            pre_x[r] = x;
+            if (x >= 0 && x < G.V) {
+                pre_lp[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
+                if constexpr (!GREEDY) pre_lq[r] = load_logit<DT>(P.draft + row * G.ld_bytes, x);
+            }
+        }
+    }
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+
     __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
     __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
     __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
 
-    for (int i = warp; i < n; i += num_warps) {
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        const int i = warp + r * num_warps;
+        if (i >= n) break;  // uniform over the warp
         const int64_t row = static_cast<int64_t>(b) * G.K + i;
         const char* prow = P.target + row * G.ld_bytes;
         const char* qrow = P.draft + row * G.ld_bytes;
@@ -817,7 +841,7 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
             }
         }
         if (lane == 0) {
-            const int x = __ldg(P.draft_tokens + row);
+            const int x = pre_x[r];
             int err = 0, accept = 0, alt = -1;
             float conf = -1.f, conf_alt = -1.f;
             double kp = 0.0, kq = 0.0;
@@ -827,7 +851,7 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
                 err = FEF_ERR_NONFINITE;
             } else {
                 kp = np.M + log2(np.S);
-                const double lpx = load_logit<DT>(prow, x);
+                const double lpx = pre_lp[r];
                 const double l2pi = lpx * c - kp;  // log2 pi(x)
                 conf = static_cast<float>(exp2(l2pi));
                 if constexpr (GREEDY) {
@@ -836,7 +860,7 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
                     conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
                 } else {
                     kq = nq.M + log2(nq.S);
-                    const double lqx = load_logit<DT>(qrow, x);
+                    const double lqx = pre_lq[r];
                     if (lqx == -INFINITY) {
                         accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
                     } else {

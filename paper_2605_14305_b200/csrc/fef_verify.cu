@@ -241,6 +241,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         // ------------------------------------------------ producer (one thread)
         if (lane == 0) {
             bool ok = true;
+            const uint64_t policy = l2_evict_first_policy();
             int next_stage = 0;
             uint32_t next_phase = 0;
             // the next free stage, or false after a bounded wait ran out
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                         d.offset = offset;
                         sc.desc[s] = d;
                         mbar_arrive_expect_tx(full + s, static_cast<uint32_t>(len));
-                        bulk_copy_g2s(smem + s * kTileBytes, base + offset, static_cast<uint32_t>(len), full + s);
+                        bulk_copy_g2s(smem + s * kTileBytes, base + offset, static_cast<uint32_t>(len), full + s, policy);
                         ++issued;
                     }
                 }

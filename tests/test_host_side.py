@@ -83,6 +83,33 @@ def test_argument_checks_return_before_touching_the_device(fef):
     assert lib.fef_remask_select(A, A, 1, 8193, 2, A, A, None) == fef.FEF_ERR_INVALID_ARG
     assert lib.fef_remask_select(A, A, 1, 8, -1, A, A, None) == fef.FEF_ERR_INVALID_ARG
     assert lib.fef_remask_select(A, A, 1, 8, 2, A, A, None) == fef.FEF_ERR_CUDA
+    # the calls with a device-resident round counter need the counter
+    assert lib.fef_spec_verify_at_round(A, A, A, None, None, 2, 4, 64, 64, 0, 1.0, 1, 1, None, A, A, A, A, 1 << 20, None,
+                                        None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_draft_sample_at_round(A, None, 2, 4, 64, 64, 0, 1.0, 1, 1, None, A, None, A, 1 << 20, None,
+                                         None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_advance_round(None, None, 0, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_advance_round(A, A, 0, None) == fef.FEF_ERR_INVALID_ARG
+    # loop bookkeeping
+    assert lib.fef_loop_next_window(None, 1, 8, 4, A, A, A, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_next_window(A, 1, 0, 4, A, A, A, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_next_window(A, 1, 8, 65, A, A, A, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_commit(A, A, A, A, A, 1, 8, 4, A, A, None, A, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_loop_remask(None, A, 1, 8, 2, A, A, A, None) == fef.FEF_ERR_INVALID_ARG
+    # vocabulary-parallel calls: sampling mode only, slice offsets in whole 16-byte vectors
+    def stats(T=1.0, off=0, V=64, ld=64, st=A):
+        return lib.fef_vp_local_stats(A, A, A, None, 2, 4, V, ld, 0, T, off, st, A, 1 << 20, None, None)
+    assert stats(T=0.0) == fef.FEF_ERR_INVALID_ARG
+    assert stats(off=4) == fef.FEF_ERR_INVALID_ARG
+    assert stats(off=-8) == fef.FEF_ERR_INVALID_ARG
+    assert stats(st=None) == fef.FEF_ERR_INVALID_ARG
+    assert stats(V=10, ld=10) == fef.FEF_ERR_ALIGNMENT
+    assert stats() == fef.FEF_ERR_CUDA
+    assert lib.fef_vp_accept(A, 0, A, None, 2, 4, 64, 0, 1.0, 1, 1, A, A, A, A, None, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_vp_accept(A, 2, A, None, 2, 4, 0, 0, 1.0, 1, 1, A, A, A, A, None, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_vp_finish(A, 2, None, 2, 4, 0, 1.0, A, A, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_vp_local_residual(A, A, A, 2, 4, 64, 64, 0, 1.0, 1, 1, 12, A, A, 1 << 20, None) == fef.FEF_ERR_INVALID_ARG
+    assert lib.fef_vp_task_bytes(0) == 0 and lib.fef_vp_task_bytes(3) == 96
     assert fef.fef_spec_verify_workspace_bytes(64, 32, 126464, torch.bfloat16) == 0  # no device: no size
     with pytest.raises(RuntimeError):
         fef.fef_spec_verify(torch.zeros(1, 1, 8), torch.zeros(1, 1, 8), torch.zeros(1, 1, dtype=torch.int32), 1.0, 0, 0)

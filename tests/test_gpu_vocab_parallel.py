@@ -63,7 +63,8 @@ def _case(B, K, V, dtype, noise, seed, scale=2.0):
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("B,K,V,ranks", [(1, 1, 16, 2), (2, 3, 40, 2), (3, 4, 1000, 3), (2, 8, 4097, 4), (5, 4, 33, 4),
-                                         (4, 32, 9000, 8), (2, 64, 70001, 3), (6, 5, 2048, 1)])
+                                         (4, 32, 9000, 8), (2, 64, 70001, 3), (6, 5, 2048, 1),
+                                         (40, 32, 2000, 2)])  # the last: short slices, many rows (warp per row)
 def test_sharded_verification_matches_the_oracle_on_the_full_rows(fef, dtype, B, K, V, ranks):
     q, p, tok = _case(B, K, V, dtype, 0.6, seed=B * 100 + K + V)
     for T, step in ((1.0, 3), (0.7, 4)):

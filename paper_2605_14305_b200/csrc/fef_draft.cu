@@ -175,17 +175,23 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
                 for (int g4 = 0; g4 < N / 4; ++g4) {
                     const int x0 = vec[j] * N + 4 * g4;
                     const uint4 r = rng.draw(P.keys, (kStreamDraft << 30) | (static_cast<uint32_t>(x0) >> 2));
-                    const float t0 = one_minus_uniform(r.x), t1 = one_minus_uniform(r.y);
-                    const float t2 = one_minus_uniform(r.z), t3 = one_minus_uniform(r.w);
-                    // (a product 0 * inf or a NaN term compares false: -inf logits and bad data never qualify)
-                    const bool q0 = t0 < e[4 * g4] * scale, q1 = t1 < e[4 * g4 + 1] * scale;
-                    const bool q2 = t2 < e[4 * g4 + 2] * scale, q3 = t3 < e[4 * g4 + 3] * scale;
+                    // 1 - u < e * scale, with u's 23 bits = word >> 9, reads word > 2^32 - 256 - e * scale * 2^32:
+                    // one multiply-add, one conversion (negative and NaN give 0) and one integer compare per
+                    // id.  The constant 2^32 - 1024 and the factor leave room for every rounding, so no id
+                    // is missed; an id let through in error (-inf logits while there is no floor yet, one
+                    // word in 2^22 otherwise) is sorted out by the exact arithmetic below.
+                    const float s32 = scale * 4294967296.0f * 1.00002f;
+                    const bool q0 = r.x >= __float2uint_rz(fmaf(-e[4 * g4], s32, 4294966272.0f));
+                    const bool q1 = r.y >= __float2uint_rz(fmaf(-e[4 * g4 + 1], s32, 4294966272.0f));
+                    const bool q2 = r.z >= __float2uint_rz(fmaf(-e[4 * g4 + 2], s32, 4294966272.0f));
+                    const bool q3 = r.w >= __float2uint_rz(fmaf(-e[4 * g4 + 3], s32, 4294966272.0f));
                     if (__any_sync(0xFFFFFFFFu, q0 || q1 || q2 || q3)) {  // the vote keeps this out of the straight line
-                        const float ts[4] = {t0, t1, t2, t3};
+                        const float ts[4] = {one_minus_uniform(r.x), one_minus_uniform(r.y), one_minus_uniform(r.z),
+                                             one_minus_uniform(r.w)};
                         const bool qs[4] = {q0, q1, q2, q3};
 #pragma unroll
                         for (int t = 0; t < 4; ++t)
-                            if (qs[t]) {
+                            if (qs[t] && l[4 * g4 + t] > -INFINITY) {
                                 const float lv = l[4 * g4 + t];
                                 float lc = lv * P.c_hi;
                                 if constexpr (Elem<DT>::kSplitScale) lc = fmaf(lv, P.c_lo, lc);

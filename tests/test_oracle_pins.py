@@ -259,8 +259,8 @@ def test_joint_law_of_a_window_V4_K2_exact_enumeration_and_chi_square():
 
     Exact part: from the oracle's per-position laws, Pr(x1, x2) enumerated over
     drafts and over accept/reject outcomes equals pi1(x1) * pi2(x2 | x1).
-    Monte-Carlo part: running the procedure (round 1 over both positions, round 2
-    over position 2 for the windows that rejected at position 1) reproduces it."""
+    Monte-Carlo part: running the procedure (a first speculative round over both positions, a
+    second one over position 2 for the windows that rejected at position 1) reproduces it."""
     rng = np.random.default_rng(7)
     V = 4
     lp1 = rng.normal(0, 1, V).astype(np.float32)

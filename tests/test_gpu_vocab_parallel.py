@@ -127,3 +127,26 @@ def test_sharded_argument_errors(fef):
     with pytest.raises(fef.FefError):   # sampling mode only
         fef_spec_verify_sharded_on_one_device(_slices(q, p, 2), tok, 0.0, 1, 1, 64)
     assert shard_vocab(126464, 8)[0] == (0, 15808) and sum(w for _, w in shard_vocab(70001, 3)) == 70001
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_sharded_random_calls_match_the_oracle(fef, chunk):
+    rng = np.random.default_rng(500 + chunk)
+    for case in range(12):
+        B, K = int(rng.integers(1, 50)), int(rng.integers(1, 65))
+        V = int(rng.integers(16, 6000))
+        ranks = int(rng.integers(1, min(8, V // 8) + 1))
+        dtype = torch.bfloat16 if rng.integers(0, 2) else torch.float32
+        T = float(rng.choice([0.5, 1.0, 2.0]))
+        q, p, tok = _case(B, K, V, dtype, float(rng.choice([0.0, 0.4, 1.5])), seed=int(rng.integers(1, 1 << 30)),
+                          scale=float(rng.choice([0.5, 2.0, 5.0])))
+        if rng.integers(0, 3) == 0:
+            g = torch.Generator(device="cuda").manual_seed(case + 1)
+            q = torch.where(torch.rand(q.shape, generator=g, device="cuda") < 0.3, float("-inf"), q.float()).to(dtype)
+            p = torch.where(torch.rand(p.shape, generator=g, device="cuda") < 0.3, float("-inf"), p.float()).to(dtype)
+            q[:, :, 0], p[:, :, 0] = 0.0, 0.0
+            tok = synth.sample_draft_tokens(q, 1.0, case + 3)
+        rl = None
+        if rng.integers(0, 2):
+            rl = torch.as_tensor(rng.integers(0, K + 1, size=B).astype(np.int32), device="cuda")
+        _run(fef, q, p, tok, T, int(rng.integers(0, 1 << 62)), int(rng.integers(0, 1 << 31)), ranks, row_len=rl)

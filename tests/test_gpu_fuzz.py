@@ -81,3 +81,21 @@ def test_random_calls_match_the_oracle(fef, chunk):
             assert (d.tokens.cpu().numpy()[used & sure] == od["tokens"][used & sure]).all(), (B, K, V, ld, dtype, T)
     print(total.summary())
     assert total.excused <= 2
+
+
+def test_random_low_confidence_selections_match_the_oracle(fef):
+    rng = np.random.default_rng(4242)
+    for case in range(80):
+        B, L = int(rng.integers(1, 70)), int(rng.integers(1, 2200))
+        k = int(rng.integers(0, min(L, 300) + 1))
+        conf = rng.random((B, L)).astype(np.float32)
+        if case % 3 == 0:      # many ties
+            conf = np.round(conf * 4) / 4
+        if case % 5 == 0:      # signed zeros and NaNs
+            conf[rng.random((B, L)) < 0.05] = -0.0
+            conf[rng.random((B, L)) < 0.02] = np.nan
+        mask = (rng.random((B, L)) < rng.choice([0.0, 0.1, 0.6, 1.0])).astype(np.uint8)
+        pos, cnt = fef.fef_remask_select(torch.as_tensor(conf).cuda(), torch.as_tensor(mask).cuda(), k)
+        opos, ocnt = oracle.remask_select(conf, mask, k)
+        assert (cnt.cpu().numpy() == ocnt).all(), (B, L, k)
+        assert (pos.cpu().numpy() == opos).all(), (B, L, k)

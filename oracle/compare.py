@@ -15,6 +15,7 @@ import numpy as np
 
 MARGIN = 1e-6
 CONF_RTOL = 1e-5
+F32_SUBNORMAL_STEP = 2.0 ** -149   # spacing of binary32 numbers below 2^-126
 
 
 @dataclass
@@ -39,15 +40,39 @@ class ParityReport:
     def ok(self) -> bool:
         return not self.mismatches
 
+    @property
+    def within_budget(self) -> bool:
+        """Excused windows must stay below 1e-5 of the draws made; with fewer than 1e5 draws that
+        means none at all."""
+        return self.excused == 0 if self.draws < 100000 else self.excused < 1e-5 * self.draws
+
     def summary(self) -> str:
         return ("windows=%d draws=%d near_margin=%d excused=%d mismatches=%d max_conf_rel_err=%.3g"
                 % (self.windows, self.draws, self.near_margin, self.excused, len(self.mismatches),
                    self.max_conf_rel_err))
 
 
-def compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int = 0) -> ParityReport:
+# Everything compared in this process, summed: a test session checks the excuse budget on it.
+LEDGER = ParityReport()
+
+
+def compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int = 0,
+                   ledger: bool = True) -> ParityReport:
     """``got_*``: arrays of the implementation under test for the same windows as ``ref``
-    (the dict returned by ``oracle.spec_verify``)."""
+    (the dict returned by ``oracle.spec_verify``).  The result is also added to ``LEDGER``
+    unless ``ledger`` is false."""
+    rep = _compare_verify(got_accept_len, got_tokens, got_conf, ref, batch_offset)
+    if ledger:
+        LEDGER.windows += rep.windows
+        LEDGER.draws += rep.draws
+        LEDGER.excused += rep.excused
+        LEDGER.near_margin += rep.near_margin
+        LEDGER.mismatches += rep.mismatches[:3]
+        LEDGER.max_conf_rel_err = max(LEDGER.max_conf_rel_err, rep.max_conf_rel_err)
+    return rep
+
+
+def _compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int) -> ParityReport:
     ga = np.asarray(got_accept_len)
     gt = np.asarray(got_tokens)
     gc = np.asarray(got_conf, dtype=np.float64)
@@ -90,8 +115,10 @@ def compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset
             denom = np.maximum(np.abs(r), 1e-300)
             rel = np.abs(g - r) / denom
             rel = np.where((r == 0) & (g == 0), 0.0, rel)
-            # binary32 output: a confidence below the smallest normal float cannot carry 1e-5
-            rel = np.where(np.abs(r) < 1e-37, np.minimum(rel, np.abs(g - r) / 1e-37 * CONF_RTOL), rel)
+            # the confidences under test are binary32 numbers: a difference of at most one step of
+            # the binary32 grid at that magnitude (a subnormal step for confidences below 2^-126) is
+            # rounding of the output type, not of the method
+            rel = np.where(np.abs(g - r) <= F32_SUBNORMAL_STEP, 0.0, rel)
             worst = float(rel.max())
             rep.max_conf_rel_err = max(rep.max_conf_rel_err, worst)
             if worst > CONF_RTOL:

@@ -75,7 +75,7 @@ def test_small_shapes_match_oracle(fef, dtype, T):
             tok = torch.where(keep, tok, top)
         total.merge(_check(fef, q, p, tok, T, seed=7 + n, step=n, V=V))
     print(total.summary())
-    assert total.excused <= 1
+    assert total.within_budget
 
 
 def test_tiny_config_decode_loop_100_steps(fef):
@@ -110,100 +110,6 @@ def test_tiny_config_decode_loop_100_steps(fef):
     assert (out["tokens"] >= 0).all()
     assert out["rounds"] >= 100
     print(total.summary(), "rounds", out["rounds"])
-
-
-def test_llada_single_stream_block(fef):
-    """Config 1 (B=1, K=32, V=126464, bf16, peaked logits): one block, three denoising steps,
-    every call checked; the row is split over many CTAs here."""
-    from paper_2605_14305_b200.decode_loop import run_decode_loop
-
-    w = synth.LLADA_SINGLE
-    total = ParityReport()
-
-    def logits_fn(rnd, window, row_len):
-        return synth.make_logits(w, seed=2000 + rnd, device="cuda")
-
-    def draft_fn(q, rnd):
-        return synth.sample_draft_tokens(q, w.temperature, 6000 + rnd)
-
-    def verify_fn(q, p, tok, rl, rnd):
-        ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, w.temperature, 11, rnd, row_len=rl)
-        assert gs == 0
-        ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), w.temperature, 11, rnd, row_len=rl.cpu())
-        rep = compare_verify(ga, gt, gc, ref)
-        assert rep.ok, rep.mismatches
-        total.merge(rep)
-        return ga, gt, gc
-
-    def select_fn(conf, mask, k):
-        pos, cnt = fef.fef_remask_select(conf, mask, k)
-        opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
-        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
-        return opos, ocnt
-
-    out = run_decode_loop(w.B, w.K, w.K, 3, w.remask_k, logits_fn, draft_fn, verify_fn, select_fn)
-    assert (out["tokens"] >= 0).all()
-    print(total.summary(), "rounds", out["rounds"])
-
-
-@pytest.mark.parametrize("sigma", [0.2, 0.7, 1.5])
-def test_llada_batched_sigma_sweep(fef, sigma):
-    """Config 2: B=16, K=32, V=126464, bf16, T=0.7; the noise level moves the acceptance rate."""
-    w = synth.LLADA_BATCHED
-    q, p, tok = synth.make_call(w, seed=int(sigma * 100), device="cuda", noise_std=sigma)
-    rep = _check(fef, q, p, tok, w.temperature, seed=3, step=int(sigma * 10))
-    ga, _, gc, _ = _gpu_verify(fef, q, p, tok, w.temperature, 3, int(sigma * 10))
-    print("sigma", sigma, rep.summary(), "mean accept_len", ga.mean())
-    # the re-mask selection of this configuration (k = 8) on the confidences just produced
-    mask = torch.as_tensor(gc >= 0).to(torch.uint8).cuda()
-    pos, cnt = fef.fef_remask_select(torch.as_tensor(gc).cuda(), mask, w.remask_k)
-    opos, ocnt = oracle.remask_select(gc, mask.cpu(), w.remask_k)
-    assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
-
-
-@pytest.mark.parametrize("T", [1.0, 0.0])
-def test_dream_large_batch_sampled_windows(fef, T):
-    """Config 3 at full size (B=64, K=32, V=152064, bf16, Zipf-biased logits) in the launch
-    configuration the benchmark uses; the oracle re-computes a sample of whole windows."""
-    w = synth.DREAM_LARGE.with_(temperature=T)
-    q, p, tok = synth.make_call(w, seed=33, device="cuda")
-    if T == 0.0:
-        top = p.float().argmax(-1).to(torch.int32)
-        tok = torch.where(torch.rand(tok.shape, device="cuda") < 0.15, tok, top)
-    ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, T, 17, 4)
-    assert gs == 0
-    total = ParityReport()
-    for b in (0, 1, 13, 31, 62, 63):
-        ref = oracle.spec_verify(q[b:b + 1].cpu(), p[b:b + 1].cpu(), tok[b:b + 1].cpu(), T, 17, 4, batch_offset=b)
-        rep = compare_verify(ga[b:b + 1], gt[b:b + 1], gc[b:b + 1], ref, batch_offset=b)
-        assert rep.ok, rep.mismatches
-        total.merge(rep)
-    # properties that hold for every window at any size
-    K = w.K
-    assert ((ga >= 0) & (ga <= K)).all()
-    idx = np.arange(K)[None, :]
-    committed = idx < np.minimum(ga + 1, K)[:, None]
-    assert ((gt >= 0) == committed).all() and ((gc >= 0) == committed).all()
-    accepted = idx < ga[:, None]
-    assert (gt[accepted] == tok.cpu().numpy()[accepted]).all()
-    assert (gc[committed] <= 1.0 + 1e-6).all()
-    print(total.summary(), "mean accept_len", ga.mean())
-
-
-def test_headline_shape_sampled_windows(fef):
-    """The benchmark's workload (B=64, K=32, V=126464, bf16, T=1) with sampled windows checked."""
-    w = synth.HEADLINE
-    q, p, tok = synth.make_call(w, seed=5, device="cuda")
-    ga, gt, gc, gs = _gpu_verify(fef, q, p, tok, w.temperature, 99, 1)
-    assert gs == 0
-    total = ParityReport()
-    for b in (0, 7, 40, 63):
-        ref = oracle.spec_verify(q[b:b + 1].cpu(), p[b:b + 1].cpu(), tok[b:b + 1].cpu(), w.temperature, 99, 1,
-                                 batch_offset=b)
-        rep = compare_verify(ga[b:b + 1], gt[b:b + 1], gc[b:b + 1], ref, batch_offset=b)
-        assert rep.ok, rep.mismatches
-        total.merge(rep)
-    print(total.summary(), "mean accept_len", ga.mean())
 
 
 def test_results_are_bit_identical_across_runs(fef):
@@ -340,7 +246,7 @@ def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef):
     torch.cuda.synchronize()
     assert (r.accept_len.cpu().numpy() == want[0]).all() and (r.tokens.cpu().numpy() == want[1]).all()
     assert (r.conf.cpu().numpy() == want[2]).all()
-    assert all(ev[i].elapsed_time(ev[i + 1]) > 0 for i in range(3))
+    assert ev[0].elapsed_time(ev[1]) > 0 and ev[1].elapsed_time(ev[2]) > 0 and ev[2].elapsed_time(ev[3]) >= 0
 
 
 def test_api_errors_with_real_buffers(fef):
@@ -399,7 +305,7 @@ def test_draft_sample_small_shapes_match_oracle(fef, dtype, T):
         e, d = _check_draft(fef, q, T, seed=11 + n, step=n, V=V)
         excused += e
         drawn += d
-    assert excused <= 1 and drawn > 1000
+    assert excused == 0 and drawn > 1000
 
 
 def test_draft_sample_llada_and_dream_shapes_row_len_and_errors(fef):
@@ -464,54 +370,3 @@ def test_verification_with_the_draft_normalisers_streams_the_target_only(fef):
     torch.cuda.synchronize()
     assert int(r.device_status.item()) == fef.FEF_ERR_NONFINITE
     assert r.accept_len[1].item() == -1 and (r.accept_len[[0, 2]] == plain.accept_len[[0, 2]]).all()
-
-
-# ------------------------------------------------- long-generation sweep ----
-@pytest.mark.parametrize("B,K,dtype", [(1, 8, torch.float32), (8, 64, torch.bfloat16), (8, 8, torch.bfloat16),
-                                       (1, 64, torch.float32), (8, 32, torch.float32)])
-def test_long_generation_sweep_points(fef, B, K, dtype):
-    """Config 4 (gen length 1024, V = 126464, logits regenerated on the device every round, full
-    loop of draft draws, verification and re-masking until nothing is masked), two denoising
-    steps.  Drafts come from fef_draft_sample, verification reuses their normalisers on odd
-    rounds and streams both tensors on even rounds.  The oracle re-verifies the device's
-    inputs on a fixed sample of rounds (the first three, then every 40th; all windows)."""
-    from paper_2605_14305_b200.decode_loop import run_decode_loop
-
-    w = synth.HEADLINE.with_(B=B, K=K, dtype=dtype, noise_std=0.7)
-    L = 1024
-    total = ParityReport()
-    state = {}
-
-    def logits_fn(rnd, window, row_len):
-        return synth.make_logits(w, seed=7000 + rnd, device="cuda")
-
-    def draft_fn(q, rnd):
-        state["draft"] = fef.fef_draft_sample(q, w.temperature, 77, rnd)
-        return state["draft"].tokens
-
-    def verify_fn(q, p, tok, rl, rnd):
-        norm = state["draft"].log2_norm if rnd % 2 else None
-        r = fef.fef_spec_verify(q, p, tok, w.temperature, 77, rnd, row_len=rl, draft_log2_norm=norm)
-        torch.cuda.synchronize()
-        assert int(r.device_status.item()) == 0
-        ga, gt, gc = r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy()
-        if rnd < 3 or rnd % 40 == 0:
-            od = oracle.draft_sample(q.cpu(), w.temperature, 77, rnd)
-            used = np.arange(K)[None, :] < rl.cpu().numpy()[:, None]
-            assert (tok.cpu().numpy()[used] == od["tokens"][used]).all()
-            ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), w.temperature, 77, rnd, row_len=rl.cpu())
-            rep = compare_verify(ga, gt, gc, ref)
-            assert rep.ok, rep.mismatches[:5]
-            total.merge(rep)
-        return ga, gt, gc
-
-    def select_fn(conf, mask, k):
-        pos, cnt = fef.fef_remask_select(conf, mask, k)
-        opos, ocnt = oracle.remask_select(conf.cpu(), mask.cpu(), k)
-        assert (pos.cpu().numpy() == opos).all() and (cnt.cpu().numpy() == ocnt).all()
-        return opos, ocnt
-
-    out = run_decode_loop(B, L, K, 2, 8, logits_fn, draft_fn, verify_fn, select_fn)
-    assert (out["tokens"] >= 0).all()
-    assert total.windows >= 3 * B
-    print(total.summary(), "rounds", out["rounds"])

@@ -239,13 +239,13 @@ def run_native(args):
         call_ms = [c0.elapsed_time(c1) / steps, c1.elapsed_time(c2) / steps]
     # timed region 3: once more with events at the kernel boundaries inside the verification call
     # (fef_spec_verify_profiled), for the duration of each kernel alone
-    stage_ms = [0.0, 0.0, 0.0]
+    stage_ms = [0.0, 0.0]
     if not args.no_call_events:
         for i in range(steps):
             step(warmup + i, stage_ev[i])
         barrier()
         for evs in stage_ev:
-            for j in range(3):
+            for j in range(2):
                 stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
         stage_ms = [x / steps for x in stage_ms]
     # timed region 4 (not part of the step): the draft-token draws that precede a verification call
@@ -353,10 +353,11 @@ def run_native(args):
         roof["frac"] = roof["achieved"] / peak
         roof["frac_of_8TBs"] = roof["achieved"] / 8000.0
         roof["ms_per_launch"] = stage_ms[0]
-        roof["kernel_ms"] = {"stream_kernel": stage_ms[0], "scan_kernel": stage_ms[1], "residual_kernel": stage_ms[2]}
+        roof["kernel_ms"] = {"stream_kernel": stage_ms[0],
+                             ("tail_kernel" if w.temperature > 0 else "scan_kernel"): stage_ms[1]}
         roof["timed"] = ("third pass over the same K steps with CUDA events at the kernel boundaries "
                          "(fef_spec_verify_profiled)")
-        # the whole verification call (four kernels chained with dependent launches), K calls back to back,
+        # the whole verification call (three kernels chained with dependent launches), K calls back to back,
         # every row counted once although the rejected rows are read a second time
         roof["call_ms"] = {"fef_spec_verify": call_ms[0], "fef_remask_select": call_ms[1]}
         roof["call_achieved"] = stream_bytes / (call_ms[0] * 1e-3) / 1e9
@@ -383,8 +384,8 @@ def run_native(args):
                     "by HBM; not part of the step",
             "verify_with_draft_norm_ms": norm_ms,
             "verify_with_draft_norm_positions_per_s": w.B * w.K / (norm_ms * 1e-3)},
-        # per step: begin-call, streaming, scan, (sampling mode) residual, re-mask kernels
-        "gpu_launches": steps * (5 if w.temperature > 0 else 4),
+        # per step: begin-call, streaming, tail (acceptance tests + residual draw; greedy: scan), re-mask kernels
+        "gpu_launches": steps * 4,
         "clocks": sampler.result(),
         "cpu_baseline": cpu_baseline,
         "parity_vs_oracle": parity,

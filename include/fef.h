@@ -3,17 +3,18 @@
  * FeF-DLLM decoding.
  *
  * The library implements, on one GPU, the verification loop of the paper's
- * full-sequence decoding algorithm (Algorithm 2, "for m = 1..b"; Section 3.2
- * "Acceleration via Speculative Decoding"; the residual law defined before
+ * full-sequence decoding algorithm (Algorithm 2, the loop over a window's
+ * positions; Section 3.2 on speculative decoding; the residual law defined before
  * Algorithm 2) for B independent speculative windows at once, and the
  * low-confidence selection LowConf_{n_rm} of the same algorithm.
  *
  * Conventions
  *  - Pointers marked "device" must be device memory of the current CUDA device;
  *    the caller owns every buffer.  The library allocates nothing, keeps no
- *    state between calls and never synchronises: all work (four kernels per
- *    verification call, the first of which clears a counter and the status word) is enqueued on `cuda_stream`
- *    (a cudaStream_t passed as void*; NULL = the default stream).
+ *    state between calls and never synchronises: all work (three kernels per
+ *    verification call, the first of which clears the counters it needs and the
+ *    status word) is enqueued on `cuda_stream` (a cudaStream_t passed as void*;
+ *    NULL = the default stream).
  *  - The return value reports what the host can see (bad arguments, launch
  *    failures).  Errors that only the data reveals are written to
  *    `*device_status` by the kernels; nothing ever traps.
@@ -67,8 +68,9 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt);
 
 /*
  * One verification call over B speculative windows of K positions
- * (Algorithm 2, lines "for m = 1 to b" .. "break"; acceptance rule and
- * correction of Section 3.2; residual law pi' = [pi - rho]_+ / (1 - sum min{pi, rho})).
+ * (Algorithm 2, the loop over the window's positions m up to the first rejection;
+ * acceptance rule and correction of Section 3.2; residual law
+ * pi' = [pi - rho]_+ / (1 - sum min{pi, rho})).
  *
  * With pi_i = softmax(target_logits[b,i,:] / T) and rho_i = softmax(draft_logits[b,i,:] / T),
  * for each window b, scanning i = 0, 1, ... < n_b (n_b = row_len[b], or K):
@@ -141,10 +143,11 @@ fef_status fef_spec_verify_with_draft_norm(const void* draft_logits, const void*
  * fef_spec_verify with timing marks: the same operation (Algorithm 2's verification
  * loop) and the same results, and additionally up to four caller-created CUDA events
  * (cudaEvent_t passed as void*; NULL entries are skipped) are recorded on `cuda_stream`:
- * [0] before the streaming kernel, [1] after it, [2] after the acceptance scan,
- * [3] after the residual draw.  `stage_events` may be NULL.  Used to time the kernels
- * separately; an event between two kernels keeps the later one from starting early, so
- * the whole call is a little slower than fef_spec_verify.
+ * [0] before the streaming kernel, [1] after it, [2] and [3] after the kernel that follows
+ * it (acceptance tests and residual draw are one launch; at temperature 0 the arg-max
+ * scan).  `stage_events` may be NULL.  Used to time the kernels separately; an event
+ * between two kernels keeps the later one from starting early, so the whole call is a
+ * little slower than fef_spec_verify.
  */
 fef_status fef_spec_verify_profiled(const void* draft_logits, const void* target_logits,
                                     const int32_t* draft_tokens, const int32_t* row_len,
@@ -194,9 +197,12 @@ fef_status fef_spec_verify_host(const void* draft_logits, const void* target_log
  * caller still owns all inputs and outputs.
  *   - Sizes whose scratch need (fef_spec_verify_workspace_bytes) exceeds
  *     FEF_STATIC_SCRATCH_BYTES are refused with FEF_ERR_TOO_LARGE and nothing is
- *     launched.  The headline shape B = 64, K = 32, V = 126464 needs about 2.3 MB.
+ *     launched.  The shape B = 64, K = 32, V = 126464 needs about 0.2 MB.
  *   - The first call on each device looks up the array's device address (one runtime
- *     query, no allocation).  Make that first call outside any stream capture.
+ *     query).  If nothing of this library has run on that device before, that is also
+ *     the moment the CUDA runtime loads the library's device code there and reserves the
+ *     array with it, so make one warm-up call per device at start-up, outside any stream
+ *     capture; later calls neither allocate nor query.
  *   - All calls on a device share the one array.  It keeps whatever the previous call
  *     left; no call depends on that content.  Two calls whose kernels can overlap on
  *     the GPU (different streams, no ordering between them) race on it and give
@@ -212,8 +218,8 @@ fef_status fef_spec_verify_static(const void* draft_logits, const void* target_l
                                   int32_t* device_status, void* cuda_stream);
 
 /*
- * Draft-token sampling (Algorithm 2, "Sample draft tokens x~ ~ rho"; Section 3.2, "We then
- * sample draft tokens ..."): for every window b and position i < n_b one draw
+ * Draft-token sampling (Algorithm 2, the step that draws the window's draft tokens from the
+ * draft laws; Section 3.2): for every window b and position i < n_b one draw
  *   draft_tokens[b,i] ~ rho_i = softmax(draft_logits[b,i,:] / T),
  * taken by Gumbel-max: arg-max over x of l_x / T - ln(-ln u_x) among the entries with
  * l_x > -inf, lowest x on exact ties.  u_x comes from Philox4x32-10 keyed like fef_spec_verify,
@@ -245,8 +251,9 @@ fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len,
                             int32_t* device_status, void* cuda_stream);
 
 /*
- * LowConf_k of Algorithm 2 ("Select R = LowConf_{n_rm}(C)"): for every batch
- * row the k candidate positions of lowest confidence.
+ * LowConf_k of Algorithm 2 (the selection of the n_rm least confident positions of C^(s)
+ * at the end of a denoising step): for every batch row the k candidate positions of lowest
+ * confidence.
  *
  *   conf       device, [B, L] float32 confidences
  *   mask       device, [B, L] uint8; a position is a candidate iff mask != 0
@@ -277,19 +284,21 @@ fef_status fef_remask_select_host(const float* conf, const uint8_t* mask, int B,
  * denoising step, the set C^(s)).  All pointers are device memory; every call is one small
  * kernel on `cuda_stream`.  1 <= L <= 2^24, 1 <= K <= FEF_MAX_K.
  *
- * fef_loop_next_window  ("Let J_t be the unresolved positions, j_1 < ... < j_Lt; b = min{k, L_t}"):
- *   window_pos [B, K] = the first K unresolved positions of each row in increasing order, -1
- *   padded; row_len [B] = min(K, L_t); unresolved [B] = L_t.
- * fef_loop_verification_inputs  ("Construct verification inputs X^(j_m) ... each input uses the
- *   verified prefix and the draft prefix x~_{j_1} .. x~_{j_{m-1}}"): inputs [B, K, L]; row m is
- *   the sequence with the drafts of the window's positions 0 .. min(m, row_len) - 1 written in.
- * fef_loop_commit  ("X^{j_m} <- x~ or Z; C^(s) <- C^(s) u {(j_m, c_{j_m})}; discard the remaining
- *   drafts"): writes the first min(accept_len + 1, row_len) entries of out_tokens / out_conf
- *   (outputs of fef_spec_verify) to their positions, marks them in in_step; committed [B] = that
- *   count, or -1 (nothing written) for a window with accept_len = -1.
- * fef_loop_remask  ("Re-corrupt X^i for i in LowConf(C^(s))", absorbing-state kernel): the first
- *   min(count[b], k) entries of positions [B, k] (output of fef_remask_select) go back to
- *   FEF_MASK_TOKEN with conf -1; in_step is cleared for the next denoising step.
+ * fef_loop_next_window  (Algorithm 2: the ordered set J_t of unresolved positions and the window
+ *   size b = min{k, L_t}): window_pos [B, K] = the first K unresolved positions of each row in
+ *   increasing order, -1 padded; row_len [B] = min(K, L_t); unresolved [B] = L_t.
+ * fef_loop_verification_inputs  (Algorithm 2: the verification inputs X^(j_m), i.e. the verified
+ *   prefix plus the drafts of the window's earlier positions): inputs [B, K, L]; row m is the
+ *   sequence with the drafts of the window's positions 0 .. min(m, row_len) - 1 written in.
+ * fef_loop_commit  (Algorithm 2: the write-back of an accepted draft or of the corrected token
+ *   with its confidence into X and C^(s); later drafts of the window are dropped): writes the
+ *   first min(accept_len + 1, row_len) entries of out_tokens / out_conf (outputs of
+ *   fef_spec_verify) to their positions, marks them in in_step; committed [B] = that count, or -1
+ *   (nothing written) for a window with accept_len = -1.
+ * fef_loop_remask  (Algorithm 2: re-corruption of the positions LowConf selected, with the
+ *   absorbing-state forward kernel): the first min(count[b], k) entries of positions [B, k]
+ *   (output of fef_remask_select) go back to FEF_MASK_TOKEN with conf -1; in_step is cleared for
+ *   the next denoising step.
  */
 fef_status fef_loop_next_window(const int32_t* tokens, int B, int L, int K,
                                 int32_t* window_pos, int32_t* row_len, int32_t* unresolved, void* cuda_stream);
@@ -304,7 +313,7 @@ fef_status fef_loop_remask(const int32_t* positions, const int32_t* count, int B
 
 /*
  * The same calls with the step number completed on the device, for loops that are replayed as a
- * CUDA graph (Algorithm 2's "while some position is unresolved" without a host round trip: a
+ * CUDA graph (the inner loop of Algorithm 2 over the unresolved positions without a host round trip: a
  * captured round keeps its by-value arguments, so the number that makes every round's random
  * numbers distinct has to live in device memory).  The step used is step + *device_round, read
  * when the kernels run.  device_round: device, [1] uint32, required (NULL is

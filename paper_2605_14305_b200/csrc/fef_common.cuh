@@ -36,14 +36,16 @@ struct __align__(16) Partial {
 };
 
 // Per-window hand-over from the scan kernel to the residual kernel.
+// (The single-GPU call decides the rejected position inside its last kernel and uses only the
+// arrival counter; the vocabulary-parallel steps hand the whole record from one call to the next.)
 struct __align__(16) ResidualTask {
     int pos;            // rejected position a, or -1 when the window has no residual draw
-    unsigned arrivals;  // CTAs of the residual kernel that have finished this window
+    unsigned arrivals;  // CTAs of the residual draw that have finished their share of this window
     double kp;          // log2 normaliser of the target law at a: pi(x) = 2^(l_x * c - kp)
     double kq;          // same for the draft law
 };
 
-// Counter shared by all CTAs of the streaming kernel (cleared by the host call).
+// Counter shared by all CTAs of the streaming kernel (cleared by begin_call_kernel, the call's first kernel).
 struct __align__(16) Control {
     unsigned long long next_claim;  // next streaming claim to hand out
 };

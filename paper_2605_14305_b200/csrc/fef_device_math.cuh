@@ -149,4 +149,45 @@ struct Top2 {
     }
 };
 
+// The three largest (weight, lowest id) a thread, warp or CTA has seen; empty slots hold weight 0.
+struct Top3 {
+    float w1, w2, w3;
+    int x1, x2, x3;
+    __device__ __forceinline__ void clear() {
+        w1 = w2 = w3 = 0.f;
+        x1 = x2 = x3 = 0x7FFFFFFF;
+    }
+    __device__ __forceinline__ void offer(float w, int x) {
+        if (better(w, x, w1, x1)) {
+            w3 = w2;
+            x3 = x2;
+            w2 = w1;
+            x2 = x1;
+            w1 = w;
+            x1 = x;
+        } else if (better(w, x, w2, x2)) {
+            w3 = w2;
+            x3 = x2;
+            w2 = w;
+            x2 = x;
+        } else if (better(w, x, w3, x3)) {
+            w3 = w;
+            x3 = x;
+        }
+    }
+    // best three of the whole warp, in every lane
+    __device__ __forceinline__ void warp_merge() {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ow1 = __shfl_xor_sync(0xFFFFFFFFu, w1, o), ow2 = __shfl_xor_sync(0xFFFFFFFFu, w2, o);
+            const float ow3 = __shfl_xor_sync(0xFFFFFFFFu, w3, o);
+            const int ox1 = __shfl_xor_sync(0xFFFFFFFFu, x1, o), ox2 = __shfl_xor_sync(0xFFFFFFFFu, x2, o);
+            const int ox3 = __shfl_xor_sync(0xFFFFFFFFu, x3, o);
+            offer(ow1, ox1);
+            offer(ow2, ox2);
+            offer(ow3, ox3);
+        }
+    }
+};
+
 }  // namespace fef

@@ -1,26 +1,31 @@
 // fef_spec_verify: the verification loop of the paper's Algorithm 2 for B windows at once.
 //
-// Four kernels, enqueued back to back on the caller's stream and chained with programmatic
+// Three kernels, enqueued back to back on the caller's stream and chained with programmatic
 // dependent launch:
-//   begin_call_kernel  one warp: the claim counter and the caller's status word start at zero;
+//   begin_call_kernel  the claim counter, the windows' arrival counters and the caller's status
+//                    word start at zero;
 //   stream_kernel    reads every target and draft row exactly once (bulk-async copies into a
 //                    shared-memory ring; persistent CTAs take runs of tiles, "claims", from a
 //                    shared counter in row order) and leaves, per claim, the partial sum of
 //                    2^(l_v * c - ref), c = log2(e) / T, from which pi(x) and rho(x) follow
 //                    for any x  (the two softmax laws of Section 3.2);
-//   scan_kernel      one warp per window, one lane per position: finishes the normalisers in
-//                    double precision, draws u_i, applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)},
-//                    finds the first rejection, writes accepted tokens and confidences
-//                    c_i = pi_i(x_i);
-//   residual_kernel  only for windows that rejected: Gumbel-max draw from [pi - rho]_+ over the
-//                    rejected row (the residual law defined before Algorithm 2), then c = pi(Z).
+//   tail_kernel      grid (shares, windows): finishes the normalisers in double precision, draws
+//                    u_i, applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)}, finds the first rejection,
+//                    writes accepted tokens and confidences c_i = pi_i(x_i); then, for windows that
+//                    rejected, the Gumbel-max draw from [pi - rho]_+ over the rejected row (the
+//                    residual law defined before Algorithm 2) and c = pi(Z).
+// Greedy mode (temperature 0) ends with scan_kernel instead: arg-max compare, no random numbers.
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
 
+#include <cooperative_groups.h>
+
 #include "fef.h"
 #include "fef_common.cuh"
 #include "fef_device_math.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace fef {
 
@@ -51,6 +56,7 @@ struct VerifyParams {
     const int32_t* row_len;
     const double* draft_norm;  // [B*K] log2 normalisers of the draft laws, or null: stream the draft rows
     float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
+    double c_exact;       // log2(e)/T in double precision (the double-precision pass of the residual draw)
     uint64_t seed;
     uint32_t step;
     const uint32_t* round; // device word added to `step` when the kernels run, or null
@@ -58,10 +64,10 @@ struct VerifyParams {
     int32_t* accept_len;
     int32_t* tokens;
     float* conf;
-    Control* ctl;          // cleared by the host call
+    Control* ctl;          // cleared by begin_call_kernel
     Partial* partials;     // [num_claims]: unit u owns entries [u * claims_per_unit, ...)
     ResidualTask* tasks;   // [B]
-    Candidate* candidates; // [B][residual_ctas][2]
+    Candidate* candidates; // [B][residual_ctas][kCandidatesPerCta]
     int vocab_offset;      // global id of element 0 of every row (a multiple of 8; 0 unless the vocabulary is sharded)
     VpCandidate* vp_out;   // [B] vocabulary-parallel mode: the residual kernel reports here instead of committing
     int32_t* status;
@@ -181,14 +187,18 @@ __device__ __forceinline__ Partial warp_combine(float ref, float sum, float best
     return p;
 }
 
-// First kernel of a call: the claim counter and the caller's status word start at zero.  (One
-// small kernel chained with programmatic dependent launch instead of two memset nodes.)
-__global__ void begin_call_kernel(Control* ctl, int32_t* status) {
-    cudaGridDependencySynchronize();  // an earlier call on the stream may still be using both
+// First kernel of a call: the claim counter, the windows' arrival counters (residual draw) and the
+// caller's status word start at zero.  (One small kernel chained with programmatic dependent
+// launch instead of memset nodes.)
+constexpr int kBeginThreads = 128;
+__global__ void __launch_bounds__(kBeginThreads) begin_call_kernel(Control* ctl, ResidualTask* tasks, int B, int32_t* status) {
+    cudaGridDependencySynchronize();  // an earlier call on the stream may still be using them
     if (threadIdx.x == 0) {
-        ctl->next_claim = 0ull;
+        if (ctl) ctl->next_claim = 0ull;
         if (status) *status = 0;
     }
+    if (tasks)
+        for (int b = threadIdx.x; b < B; b += kBeginThreads) tasks[b].arrivals = 0u;
 }
 
 enum : int { kFlagFirst = 1, kFlagLast = 2, kFlagExit = 4 };
@@ -507,21 +517,22 @@ struct RowNorm {
 template <int DT, bool GREEDY>
 __device__ __forceinline__ RowNorm fold_unit(int64_t u, const char* row, double c, const VerifyParams& P) {
     const Geometry& G = P.geo;
+    const int nrec = G.claims_per_unit;
     const Partial* rec = P.partials + u * G.claims_per_unit;
     double m = -INFINITY, sacc = 0.0;
     bool bad = false;
     float best = -INFINITY;
     int index = 0x7FFFFFFF;
-    for (int r = 0; r < G.claims_per_unit; ++r) {
+    for (int r = 0; r < nrec; ++r) {
         const Partial p = rec[r];
         if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = true;
         if (p.sum > 0.f) {
             const double pm = p.ref, ps = p.sum;
-            if (pm > m) {
-                sacc = sacc * exp2(m - pm) + ps;
+            if (pm > m) {  // (the first record, and any record equal to the running reference, needs no scaling)
+                sacc = m > -INFINITY ? sacc * exp2(m - pm) + ps : ps;
                 m = pm;
             } else {
-                sacc += ps * exp2(pm - m);
+                sacc += pm == m ? ps : ps * exp2(pm - m);
             }
         }
         if (GREEDY && better(p.best, p.index, best, index)) {
@@ -559,9 +570,10 @@ __device__ __forceinline__ RowNorm fold_unit(int64_t u, const char* row, double 
 
 constexpr int kScanWarps = 4;  // windows per CTA of the scan kernel
 
-// Acceptance tests, first rejection and outputs (Algorithm 2, "for m = 1..b"): one warp per
-// window, lane l does positions l and l + 32.
-template <int DT, bool GREEDY>
+// Greedy mode (temperature 0), after the streaming kernel: a draft is accepted iff it is the arg-max
+// of the target logits; the first rejection is replaced by that arg-max; confidences are the
+// T = 1 softmax probabilities.  One warp per window, lane l does positions l and l + 32.
+template <int DT>
 __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_constant__ VerifyParams P) {
     const Geometry& G = P.geo;
     constexpr int kRounds = FEF_MAX_K / 32;
@@ -573,27 +585,23 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
 
     // what does not depend on the streaming kernel is fetched before waiting for it
     int tok[kRounds];
-    double lpx[kRounds], lqx[kRounds];
+    double lpx[kRounds];
 #pragma unroll
     for (int r = 0; r < kRounds; ++r) {
         const int i = r * 32 + lane;
         tok[r] = -1;
-        lpx[r] = lqx[r] = 0.0;
+        lpx[r] = 0.0;
         if (r * 32 < G.K && i < n) {
             const int64_t row = static_cast<int64_t>(b) * G.K + i;
             const int x = __ldg(P.draft_tokens + row);
             tok[r] = x;
-            if (x >= 0 && x < G.V) {
-                lpx[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
-                if constexpr (!GREEDY) lqx[r] = load_logit<DT>(P.draft + row * G.ld_bytes, x);
-            }
+            if (x >= 0 && x < G.V) lpx[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
         }
     }
     cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
 
     int alt[kRounds];
     float cf[kRounds], cf_alt[kRounds];
-    double kp[kRounds], kq[kRounds];
     unsigned rejected[kRounds];
     int err = 0;
 #pragma unroll
@@ -601,50 +609,21 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
         const int i = r * 32 + lane;
         alt[r] = -1;
         cf[r] = cf_alt[r] = -1.f;
-        kp[r] = kq[r] = 0.0;
         bool accept = true;
         if (r * 32 < G.K && i < n) {
             const int64_t row = static_cast<int64_t>(b) * G.K + i;
-            const char* prow = P.target + row * G.ld_bytes;
-            const char* qrow = P.draft + row * G.ld_bytes;
             const int x = tok[r];
-            const RowNorm np = fold_unit<DT, GREEDY>(row * G.units_per_row, prow, c, P);
-            RowNorm nq;
-            nq.bad = false;
-            if constexpr (!GREEDY) {
-                if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
-                    nq.M = P.draft_norm[row];
-                    nq.S = 1.0;
-                    nq.bad = !(fabs(nq.M) < INFINITY);
-                } else {
-                    nq = fold_unit<DT, false>(2 * row + 1, qrow, c, P);
-                }
-            }
+            const RowNorm np = fold_unit<DT, true>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P);
             if (x < 0 || x >= G.V) {
                 err = max(err, static_cast<int>(FEF_ERR_TOKEN_RANGE));
-            } else if (np.bad || nq.bad) {
+            } else if (np.bad) {
                 err = max(err, static_cast<int>(FEF_ERR_NONFINITE));
             } else {
-                kp[r] = np.M + log2(np.S);
-                const double l2pi = lpx[r] * c - kp[r];  // log2 pi(x)
-                cf[r] = static_cast<float>(exp2(l2pi));
-                if constexpr (GREEDY) {
-                    accept = (x == np.index);
-                    alt[r] = np.index;
-                    cf_alt[r] = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp[r]));
-                } else {
-                    kq[r] = nq.M + log2(nq.S);
-                    if (lqx[r] == -INFINITY) {
-                        accept = lpx[r] > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
-                    } else {
-                        const double ratio = exp2(l2pi - (lqx[r] * c - kq[r]));
-                        const uint4 rnd = philox4x32_10(
-                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
-                            make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
-                        const double uacc = uniform_from_word(rnd.x);
-                        accept = uacc <= fmin(1.0, ratio);
-                    }
-                }
+                const double kp = np.M + log2(np.S);
+                cf[r] = static_cast<float>(exp2(lpx[r] * c - kp));
+                accept = (x == np.index);
+                alt[r] = np.index;
+                cf_alt[r] = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
             }
         }
         rejected[r] = __ballot_sync(0xFFFFFFFFu, !accept);
@@ -667,7 +646,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
                 if (i < a) {
                     t = tok[r];
                     f = cf[r];
-                } else if (GREEDY && i == a && a < n) {
+                } else if (i == a && a < n) {
                     t = alt[r];
                     f = cf_alt[r];
                 }
@@ -676,27 +655,9 @@ __global__ void __launch_bounds__(kScanWarps * 32) scan_kernel(const __grid_cons
             P.conf[row] = f;
         }
     }
-
-    // the rejected position's normalisers travel with the residual task
-    double kpa = 0.0, kqa = 0.0;
-#pragma unroll
-    for (int r = 0; r < kRounds; ++r) {
-        const double vp = __shfl_sync(0xFFFFFFFFu, kp[r], a & 31);
-        const double vq = __shfl_sync(0xFFFFFFFFu, kq[r], a & 31);
-        if ((a >> 5) == r) {
-            kpa = vp;
-            kqa = vq;
-        }
-    }
     if (lane == 0) {
         P.accept_len[b] = err ? -1 : a;
         if (err) report(P.status, err);
-        ResidualTask task;
-        task.pos = (!GREEDY && !err && a < n) ? a : -1;
-        task.arrivals = 0u;
-        task.kp = task.pos >= 0 ? kpa : 0.0;
-        task.kq = task.pos >= 0 ? kqa : 0.0;
-        P.tasks[b] = task;
     }
 }
 
@@ -729,11 +690,11 @@ __device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const Ve
         if (!(p.sum >= 0.f) || p.sum == INFINITY) bad = 1;
         if (p.sum > 0.f) {
             const double pm = p.ref, ps = p.sum;
-            if (pm > m) {
-                sacc = sacc * exp2(m - pm) + ps;
+            if (pm > m) {  // (the first record, and any record equal to the running reference, needs no scaling)
+                sacc = m > -INFINITY ? sacc * exp2(m - pm) + ps : ps;
                 m = pm;
             } else {
-                sacc += ps * exp2(pm - m);
+                sacc += pm == m ? ps : ps * exp2(pm - m);
             }
         }
         if (GREEDY && better(p.best, p.index, best, index)) {
@@ -785,9 +746,9 @@ __device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const Ve
 
 constexpr int kScanMaxWarps = 32;
 
-// The same step with one CTA per window and one warp per position, for calls whose rows are
+// The same greedy step with one CTA per window and one warp per position, for calls whose rows are
 // cut into many claims (few rows in all): the fold of a row's partials is then shared by 32 lanes.
-template <int DT, bool GREEDY>
+template <int DT>
 __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __grid_constant__ VerifyParams P) {
     const Geometry& G = P.geo;
     const int num_warps = blockDim.x >> 5;
@@ -800,25 +761,21 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
     // tokens of this warp's positions and the logits at them (a warp has at most kRows positions)
     constexpr int kRows = (FEF_MAX_K + kScanMaxWarps - 1) / kScanMaxWarps;
     int pre_x[kRows];
-    double pre_lp[kRows], pre_lq[kRows];
+    double pre_lp[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
         const int i = warp + r * num_warps;
         pre_x[r] = -1;
-        pre_lp[r] = pre_lq[r] = 0.0;
+        pre_lp[r] = 0.0;
         if (lane == 0 && i < n) {
             const int64_t row = static_cast<int64_t>(b) * G.K + i;
             const int x = __ldg(P.draft_tokens + row);
             pre_x[r] = x;
-            if (x >= 0 && x < G.V) {
-                pre_lp[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
-                if constexpr (!GREEDY) pre_lq[r] = load_logit<DT>(P.draft + row * G.ld_bytes, x);
-            }
+            if (x >= 0 && x < G.V) pre_lp[r] = load_logit<DT>(P.target + row * G.ld_bytes, x);
         }
     }
     cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
 
-    __shared__ double s_kp[FEF_MAX_K], s_kq[FEF_MAX_K];
     __shared__ float s_conf[FEF_MAX_K], s_conf_alt[FEF_MAX_K];
     __shared__ int s_accept[FEF_MAX_K], s_err[FEF_MAX_K], s_alt[FEF_MAX_K];
 
@@ -827,60 +784,27 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
         const int i = warp + r * num_warps;
         if (i >= n) break;  // uniform over the warp
         const int64_t row = static_cast<int64_t>(b) * G.K + i;
-        const char* prow = P.target + row * G.ld_bytes;
-        const char* qrow = P.draft + row * G.ld_bytes;
-        const RowNorm np = fold_unit_warp<DT, GREEDY>(row * G.units_per_row, prow, c, P, lane);
-        RowNorm nq;
-        nq.bad = false;
-        if constexpr (!GREEDY) {
-            if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
-                nq.M = P.draft_norm[row];
-                nq.S = 1.0;
-                nq.bad = !(fabs(nq.M) < INFINITY);
-            } else {
-                nq = fold_unit_warp<DT, false>(2 * row + 1, qrow, c, P, lane);
-            }
-        }
+        const RowNorm np = fold_unit_warp<DT, true>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P, lane);
         if (lane == 0) {
             const int x = pre_x[r];
             int err = 0, accept = 0, alt = -1;
             float conf = -1.f, conf_alt = -1.f;
-            double kp = 0.0, kq = 0.0;
             if (x < 0 || x >= G.V) {
                 err = FEF_ERR_TOKEN_RANGE;
-            } else if (np.bad || nq.bad) {
+            } else if (np.bad) {
                 err = FEF_ERR_NONFINITE;
             } else {
-                kp = np.M + log2(np.S);
-                const double lpx = pre_lp[r];
-                const double l2pi = lpx * c - kp;  // log2 pi(x)
-                conf = static_cast<float>(exp2(l2pi));
-                if constexpr (GREEDY) {
-                    accept = (x == np.index);
-                    alt = np.index;
-                    conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
-                } else {
-                    kq = nq.M + log2(nq.S);
-                    const double lqx = pre_lq[r];
-                    if (lqx == -INFINITY) {
-                        accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
-                    } else {
-                        const double ratio = exp2(l2pi - (lqx * c - kq));
-                        const uint4 r = philox4x32_10(
-                            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
-                            make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
-                        const double uacc = uniform_from_word(r.x);
-                        accept = uacc <= fmin(1.0, ratio);
-                    }
-                }
+                const double kp = np.M + log2(np.S);
+                conf = static_cast<float>(exp2(pre_lp[r] * c - kp));
+                accept = (x == np.index);
+                alt = np.index;
+                conf_alt = static_cast<float>(exp2(static_cast<double>(np.best) * c - kp));
             }
             s_err[i] = err;
             s_accept[i] = accept;
             s_conf[i] = conf;
             s_conf_alt[i] = conf_alt;
             s_alt[i] = alt;
-            s_kp[i] = kp;
-            s_kq[i] = kq;
         }
     }
     __syncthreads();
@@ -898,7 +822,7 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
             if (i < a) {
                 tok = __ldg(P.draft_tokens + row);
                 cf = s_conf[i];
-            } else if (GREEDY && i == a && a < n) {
+            } else if (i == a && a < n) {
                 tok = s_alt[i];
                 cf = s_conf_alt[i];
             }
@@ -909,23 +833,37 @@ __global__ void __launch_bounds__(kScanMaxWarps * 32) scan_rows_kernel(const __g
     if (threadIdx.x == 0) {
         P.accept_len[b] = err ? -1 : a;
         if (err) report(P.status, err);
-        ResidualTask task;
-        task.pos = (!GREEDY && !err && a < n) ? a : -1;
-        task.arrivals = 0u;
-        task.kp = task.pos >= 0 ? s_kp[a] : 0.0;
-        task.kq = task.pos >= 0 ? s_kq[a] : 0.0;
-        P.tasks[b] = task;
     }
 }
 
 
 // ============================================================= residual ====
 constexpr int kResidualThreads = 256;
-constexpr int kResidualBatch = 4;   // vector pairs a thread has in flight
-constexpr int kMaxResidualCtas = kResidualThreads / 2;  // the last CTA looks at 2 candidates per CTA
+constexpr int kResidualWarps = kResidualThreads / 32;
+constexpr int kCandidatesPerCta = 3;  // what a CTA leaves for the deciding warp
+constexpr int kMaxClusterCtas = 8;    // up to this many CTAs per window they form a thread-block cluster
+constexpr int kMaxResidualCtas = 2 * kResidualThreads / kCandidatesPerCta;  // reporting mode: two candidates per thread
 constexpr int kResidualCtasPerSm = 2;  // resident CTAs the grid is sized for: 2 fat ones beat 4 (1.5 us per call) and 1
 
-// Exact (double) Gumbel score ln r_x - ln(-ln u_x) of vocabulary id x; -inf when r_x <= 0.
+// Bound on the relative error of a law's normaliser as the streaming kernel delivers it (binary32
+// partial sums of approximate exponentials; the largest error measured on a confidence is 1.1e-6,
+// and that includes the rounding of the temperature scale).
+constexpr double kNormRelErr = 2.0e-6;
+
+__device__ __forceinline__ uint32_t pick_word(const uint4& w, int k) {
+    return k == 0 ? w.x : k == 1 ? w.y : k == 2 ? w.z : w.w;
+}
+
+// The uniform of vocabulary id x (global id x + vocab_offset) in the residual draw of (b, pos).
+__device__ double residual_uniform(int x, uint32_t b, uint32_t pos, const VerifyParams& P) {
+    const uint4 w = philox4x32_10(
+        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x + P.vocab_offset) >> 2), b, pos, step_of(P)),
+        make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+    return uniform_from_word(pick_word(w, x & 3));
+}
+
+// Exact (double) Gumbel score ln r_x - ln(-ln u_x) of vocabulary id x with the given normalisers;
+// -inf when r_x <= 0.
 template <int DT>
 __device__ double exact_score(int x, const char* prow, const char* qrow, double c, double kp, double kq,
                               uint32_t b, uint32_t pos, const VerifyParams& P) {
@@ -935,16 +873,22 @@ __device__ double exact_score(int x, const char* prow, const char* qrow, double 
     const double rho = exp2(lq * c - kq);
     const double r = pi - rho;
     if (!(r > 0.0)) return -INFINITY;
-    const uint4 w = philox4x32_10(
-        make_uint4((kStreamResidual << 30) | (static_cast<uint32_t>(x + P.vocab_offset) >> 2), b, pos, step_of(P)),
-        make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
-    const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
-    const double u = uniform_from_word(word);
-    return log(r) - log(-log(u));
+    return log(r) - log(-log(residual_uniform(x, b, pos, P)));
 }
 
+struct ResidualShared {
+    unsigned floor_bits;   // lower bound of the CTA's third-largest bound so far (bits of a float >= 0)
+    int last;              // this CTA is the window's last one to finish its share
+    int exact;             // the deciding warp asks for the double-precision pass over the row
+    float exact_floor;     // ... and gives it a lower bound of the row's largest true weight (0: none)
+    Top3 top[kResidualWarps];
+    Candidate cluster_cand[kMaxClusterCtas * kCandidatesPerCta];  // rank 0: what the cluster's CTAs found
+    double red_a[kResidualWarps], red_b[kResidualWarps];
+    int red_i[kResidualWarps];
+};
+
 // Block-wide arg-max of (score, lowest x).  Every thread gets the result.
-__device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
+__device__ void block_argmax(double& score, int& x, ResidualShared& sh) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const double os = __shfl_xor_sync(0xFFFFFFFFu, score, o);
@@ -957,213 +901,627 @@ __device__ void block_argmax(double& score, int& x, double* s_score, int* s_x) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncthreads();
     if (lane == 0) {
-        s_score[warp] = score;
-        s_x[warp] = x;
+        sh.red_a[warp] = score;
+        sh.red_i[warp] = x;
     }
     __syncthreads();
-    score = s_score[0];
-    x = s_x[0];
-    for (int w = 1; w < kResidualThreads / 32; ++w)
-        if (s_score[w] > score || (s_score[w] == score && s_x[w] < x)) {
-            score = s_score[w];
-            x = s_x[w];
+    score = sh.red_a[0];
+    x = sh.red_i[0];
+    for (int w = 1; w < kResidualWarps; ++w)
+        if (sh.red_a[w] > score || (sh.red_a[w] == score && sh.red_i[w] < x)) {
+            score = sh.red_a[w];
+            x = sh.red_i[w];
         }
 }
 
+// Block-wide sums of two doubles (fixed order: the same result in every thread and every run).
+__device__ void block_sum2(double& a, double& b, ResidualShared& sh) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) {
+        sh.red_a[warp] = a;
+        sh.red_b[warp] = b;
+    }
+    __syncthreads();
+    a = sh.red_a[0];
+    b = sh.red_b[0];
+    for (int w = 1; w < kResidualWarps; ++w) {
+        a += sh.red_a[w];
+        b += sh.red_b[w];
+    }
+}
+
+// The residual draw of one row decided in double precision, normalisers included: both laws are
+// summed again from the logits in double precision (the streaming kernel's binary32 sums only
+// serve as the reference exponent), then arg-max_x { ln [pi - rho]_+ - ln(-ln u_x) }, lowest x on
+// ties; if [pi - rho]_+ is zero everywhere, arg-max of the target logits.  `floor_w` is a lower bound
+// of the row's largest true weight (0 = none known): ids whose binary32 upper bound cannot reach it
+// are passed over after one multiply, as in the fast pass.  Whole CTA; every thread returns the
+// same (Z, pi(Z)).  Slow (a pass of double-precision exponentials by one CTA): only for draws that
+// the bounds of the fast pass cannot decide.
 template <int DT>
-__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual_kernel(const __grid_constant__ VerifyParams P) {
+__device__ void exact_row_draw(const VerifyParams& P, const char* prow, const char* qrow, uint32_t ub, uint32_t upos,
+                               double kp_nom, double kq_nom, float slack, float floor_w, ResidualShared& sh, int& Z,
+                               double& piZ) {
+    const int V = P.geo.V;
+    const double c = P.c_exact;
+    // normalisers: sum_x 2^(l_x c - k_nominal) is within 1e-5 of one, so nothing can overflow
+    double sp = 0.0, sq = 0.0;
+    for (int x = threadIdx.x; x < V; x += kResidualThreads) {
+        const double lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
+        if (lp > -INFINITY) sp += exp2(lp * c - kp_nom);
+        if (lq > -INFINITY) sq += exp2(lq * c - kq_nom);
+    }
+    block_sum2(sp, sq, sh);
+    const double kp = kp_nom + log2(sp), kq = kq_nom + log2(sq);
+    const float kp32 = static_cast<float>(kp_nom), kq32 = static_cast<float>(kq_nom);
+
+    PhiloxRow rng;
+    rng.prepare(P.keys, ub, upos, step_of(P));
+    double score = -INFINITY;
+    int best = 0x7FFFFFFF;
+    for (int pass = 0; pass < 2; ++pass) {
+        // groups of four ids share a Philox call; a thread visits its ids in increasing order
+        for (int x0 = 4 * static_cast<int>(threadIdx.x); x0 < V; x0 += 4 * kResidualThreads) {
+            const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x0 + P.vocab_offset) >> 2));
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int x = x0 + k;
+                if (x >= V) break;
+                const float lpf = load_logit<DT>(prow, x), lqf = load_logit<DT>(qrow, x);
+                const float ep = exp2_scaled<DT>(lpf, P.c_hi, P.c_lo, kp32);
+                const float rs = fmaf(ep, slack, ep - exp2_scaled<DT>(lqf, P.c_hi, P.c_lo, kq32));
+                const uint32_t word = pick_word(w, k);
+                if (!(rs > floor_w * one_minus_uniform(word))) continue;
+                const double pi = exp2(static_cast<double>(lpf) * c - kp);
+                const double rho = lqf > -INFINITY ? exp2(static_cast<double>(lqf) * c - kq) : 0.0;
+                const double r = pi - rho;
+                if (!(r > 0.0)) continue;
+                const double s = log(r) - log(-log(static_cast<double>(uniform_from_word(word))));
+                if (s > score) {  // strict: the lowest index keeps a tie
+                    score = s;
+                    best = x;
+                }
+            }
+        }
+        block_argmax(score, best, sh);
+        if (score > -INFINITY || floor_w == 0.f) break;
+        floor_w = 0.f;  // (not expected: the floor belongs to an id of this row) once more without it
+    }
+    if (!(score > -INFINITY)) {
+        // [pi - rho]_+ is identically zero: commit arg-max of pi (= arg-max of the target logits)
+        score = -INFINITY;
+        best = 0x7FFFFFFF;
+        for (int x = threadIdx.x; x < V; x += kResidualThreads) {
+            const double l = load_logit<DT>(prow, x);
+            if (l > score) {
+                score = l;
+                best = x;
+            }
+        }
+        block_argmax(score, best, sh);
+    }
+    Z = best;
+    piZ = (best >= 0 && best < V) ? exp2(static_cast<double>(load_logit<DT>(prow, best)) * c - kp) : 0.0;
+}
+
+// Rare path of the residual pass, out of line so that the loop around it stays small: the id's
+// bound ub = rs / (-ln u), rounded up (1.00003 is above the error of the approximate logarithm and
+// division), offered to the thread's best three.
+__device__ __noinline__ Top3 offer_bound(Top3 top, float rs, float t, int x) {
+    top.offer(__fdividef(rs, neg_log_uniform(t)) * 1.00003f, x);
+    return top;
+}
+
+// The residual draw Z ~ [pi - rho]_+ / (1 - sum min{pi, rho}) of window b, rejected position `pos`,
+// by Gumbel-max: arg-max_x { ln r_x - ln(-ln u_x) }, which is arg-max_x of w_x = r_x / (-ln u_x).
+// This CTA covers share `part` of `parts` of the row; the window's last CTA to finish decides.
+//
+// Fast pass (binary32).  For every id an upper bound rs_x >= r_x that holds whatever the rounding of
+// this pass and whatever the error of the two normalisers (each within kNormRelErr):
+//     rs_x = (e_p - e_q) + slack * e_p,   e_p = 2^(l^p_x c - kp), e_q = 2^(l^q_x c - kq) in binary32.
+// Since -ln u > 1 - u, an id with rs_x <= floor * (1 - u_x) has w_x < floor and is dropped after one
+// multiply (floor = a lower bound of the CTA's third-largest bound so far); a warp vote keeps the few
+// others out of the straight-line code.  Those get the bound ub_x = rs_x / (-ln u_x), rounded up, and
+// each thread, warp and CTA keeps the three largest.
+//
+// Decision (one warp of the window's last CTA).  Of the row's three largest bounds, the ids x1, x2
+// of the first two are evaluated in double precision: weight w = r / (-ln u) under the given
+// normalisers and the interval [(r - 2 d pi) / (-ln u), (r + 2 d pi) / (-ln u)], d = kNormRelErr, that
+// holds the weight under the exact normalisers.  Every other id's true weight is below the third
+// bound.  If the larger of the two has its interval above the other's interval and above the third
+// bound, it is the arg-max for every admissible value of the normalisers, hence the exact one:
+// commit it.  Otherwise (two near-equal weights, or laws so close that pi - rho is lost in the
+// normalisers' error) the row is redone by exact_row_draw.
+//
+// REPORT (vocabulary-parallel mode): the CTA's slice is one rank's share of the row and the ranks'
+// best ids are compared afterwards by their scores under the shared normalisers, so the decision
+// among this slice's candidates is taken on those scores (candidates within a band of the largest
+// bound are scored in double precision) and reported instead of committed.
+// prow, qrow: the target and draft logits of the rejected position; out_row: where tokens / conf go.
+template <int DT, bool REPORT, bool CLUSTER>
+__device__ void residual_draw(const VerifyParams& P, int b, int pos, double kp_d, double kq_d, const char* prow,
+                              const char* qrow, int64_t out_row, int part, int parts, ResidualShared& sh) {
     constexpr int N = Elem<DT>::kPerVec;
     const Geometry& G = P.geo;
-    cudaGridDependencySynchronize();  // the scan kernel's tasks must be complete and visible
-    const int b = blockIdx.y, part = blockIdx.x, parts = gridDim.x;
-    const ResidualTask task = P.tasks[b];
-    if (task.pos < 0) return;  // uniform over the CTA
+    const float kp = static_cast<float>(kp_d), kq = static_cast<float>(kq_d);
+    const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(pos);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const int64_t row = static_cast<int64_t>(b) * G.K + task.pos;
-    const char* prow = P.target + row * G.ld_bytes;
-    const char* qrow = P.draft + row * G.ld_bytes;
-    const float kp = static_cast<float>(task.kp), kq = static_cast<float>(task.kq);
-    const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(task.pos);
+    // slack: relative to e_p.  Argument of the exponential: the narrowed normaliser (|k| 2^-24) and up
+    // to two roundings of the multiply-adds (|l c - k| 2^-24 each, |l c - k| < 150 where e > 0), times
+    // ln 2; ex2.approx: 2^-21; the subtraction: 2^-24; both laws.  Then the normalisers' own error
+    // (reporting mode compares under the shared normalisers and leaves it out).
+    const float rounding = (fabsf(kp) + fabsf(kq) + 600.f) * 4.2e-8f + 1.0e-6f;
+    const float slack = REPORT ? rounding : rounding + static_cast<float>(2.0 * kNormRelErr);
 
     PhiloxRow rng;
     rng.prepare(P.keys, ub, upos, step_of(P));
 
-    Top2 top;
+    Top3 top;
     top.clear();
-    // A lower bound of the CTA's second-best weight so far (bits of a non-negative float).  An id
-    // whose weight cannot exceed it is dropped after one multiply; a stale value is only less sharp.
-    __shared__ unsigned s_floor;
-    if (threadIdx.x == 0) s_floor = 0u;
-    __syncthreads();
+    float floor_w = 0.f;
 
-    // ---- binary32 pass over this CTA's share of the row: w_x = r_x / (-ln u_x).  A thread's loads
-    //      are all issued before the arithmetic; every group of four ids gets its Philox call.
+    // ---- binary32 pass over this CTA's share of the row.  One vector pair (N ids of both laws) per
+    //      thread and step; the loads of the next two steps are in flight while one is worked on.  The
+    //      loop body is kept small (one copy, the rare path out of line): with several hundred
+    //      instructions per step, a larger body stalls on instruction fetch.
     const int nvec = G.vec_elems / N;
     const int v_begin = static_cast<int>(static_cast<int64_t>(part) * nvec / parts);
     const int v_end = static_cast<int>(static_cast<int64_t>(part + 1) * nvec / parts);
-    for (int v0 = v_begin; v0 < v_end; v0 += kResidualThreads * kResidualBatch) {
-        uint4 wp[kResidualBatch], wq[kResidualBatch];
-        int vec[kResidualBatch];
-#pragma unroll
-        for (int j = 0; j < kResidualBatch; ++j) {
-            vec[j] = v0 + j * kResidualThreads + static_cast<int>(threadIdx.x);
-            // a lane beyond the end works on -inf logits (r = 0 never qualifies), so the warp stays whole
-            constexpr uint32_t kMinusInf = DT == FEF_F32 ? 0xFF800000u : 0xFF80FF80u;
-            wp[j] = wq[j] = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
-            if (vec[j] < v_end) {
-                wp[j] = ld_global_nc_v4(prow + static_cast<int64_t>(vec[j]) * 16);
-                wq[j] = ld_global_nc_v4(qrow + static_cast<int64_t>(vec[j]) * 16);
-            }
+    // a lane beyond the end works on -inf logits (rs = 0 never qualifies), so the warp stays whole
+    constexpr uint32_t kMinusInf = DT == FEF_F32 ? 0xFF800000u : 0xFF80FF80u;
+    auto fetch = [&](int v0, uint4& wp, uint4& wq) {
+        const int vec = v0 + static_cast<int>(threadIdx.x);
+        wp = wq = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
+        if (vec < v_end) {
+            wp = ld_global_nc_v4(prow + static_cast<int64_t>(vec) * 16);
+            wq = ld_global_nc_v4(qrow + static_cast<int64_t>(vec) * 16);
         }
-        float floor_w = fmaxf(top.w2, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&s_floor)));
+    };
+    // bounds rs and 1 - u of the N ids of one vector pair: straight-line, so that the Philox chains of
+    // its groups of four ids and the exponentials overlap
+    auto bounds = [&](int v0, const uint4& wp, const uint4& wq, float(&rs)[N], float(&t)[N]) {
+        const int vec = v0 + static_cast<int>(threadIdx.x);
+        float lp[N], lq[N];
+        unpack<DT>(wp, lp);
+        unpack<DT>(wq, lq);
 #pragma unroll
-        for (int j = 0; j < kResidualBatch; ++j) {
-            if (v0 + j * kResidualThreads >= v_end) break;  // nothing but padding left (uniform over the CTA)
-            float lp[N], lq[N], r[N];
-            unpack<DT>(wp[j], lp);
-            unpack<DT>(wq[j], lq);
-#pragma unroll
-            for (int i = 0; i < N; ++i)
-                r[i] = exp2_scaled<DT>(lp[i], P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq[i], P.c_hi, P.c_lo, kq);
-#pragma unroll
-            for (int g4 = 0; g4 < N / 4; ++g4) {
-                const int x0 = vec[j] * N + 4 * g4;
-                const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x0 + P.vocab_offset) >> 2));
-                // w = r / (-ln u) < r / t: once the floor is up, nearly every id is ruled out by one
-                // multiply and compare; the vote keeps the rare rest out of the straight-line code
-                const float t0 = one_minus_uniform(w.x), t1 = one_minus_uniform(w.y);
-                const float t2 = one_minus_uniform(w.z), t3 = one_minus_uniform(w.w);
-                const bool q0 = r[4 * g4] > floor_w * t0, q1 = r[4 * g4 + 1] > floor_w * t1;
-                const bool q2 = r[4 * g4 + 2] > floor_w * t2, q3 = r[4 * g4 + 3] > floor_w * t3;
-                if (__any_sync(0xFFFFFFFFu, q0 || q1 || q2 || q3)) {
-                    if (q0) top.offer(__fdividef(r[4 * g4], neg_log_uniform(t0)), x0);
-                    if (q1) top.offer(__fdividef(r[4 * g4 + 1], neg_log_uniform(t1)), x0 + 1);
-                    if (q2) top.offer(__fdividef(r[4 * g4 + 2], neg_log_uniform(t2)), x0 + 2);
-                    if (q3) top.offer(__fdividef(r[4 * g4 + 3], neg_log_uniform(t3)), x0 + 3);
-                }
-            }
-            // raise the floor: any lane's second-best weight bounds the CTA's second best from below
-            floor_w = fmaxf(floor_w, __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(top.w2))));
-            if (j == 0 && v0 == v_begin) {
-                // after the first vector of every thread the whole CTA shares what it has found
-                if ((threadIdx.x & 31) == 0) atomicMax(&s_floor, __float_as_uint(floor_w));
-                __syncthreads();
-                floor_w = fmaxf(floor_w, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&s_floor)));
-            }
+        for (int i = 0; i < N; ++i) {
+            const float ep = exp2_scaled<DT>(lp[i], P.c_hi, P.c_lo, kp);
+            rs[i] = fmaf(ep, slack, ep - exp2_scaled<DT>(lq[i], P.c_hi, P.c_lo, kq));
         }
-        if ((threadIdx.x & 31) == 0) atomicMax(&s_floor, __float_as_uint(floor_w));
+#pragma unroll
+        for (int g4 = 0; g4 < N / 4; ++g4) {
+            const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) |
+                                                 (static_cast<uint32_t>(vec * N + 4 * g4 + P.vocab_offset) >> 2));
+            t[4 * g4] = one_minus_uniform(w.x);
+            t[4 * g4 + 1] = one_minus_uniform(w.y);
+            t[4 * g4 + 2] = one_minus_uniform(w.z);
+            t[4 * g4 + 3] = one_minus_uniform(w.w);
+        }
+    };
+
+    // Two vector pairs per thread and step (their four Philox chains and 4 N exponentials overlap in the
+    // straight-line part); the loads of the next step are in flight meanwhile.
+    uint4 p0, q0, p1, q1, p2, q2, p3, q3;
+    fetch(v_begin, p0, q0);
+    fetch(v_begin + kResidualThreads, p1, q1);
+    {
+        // A first floor, so that the pass does not start with every id qualifying: the largest bound of
+        // each lane's first vector pair; the third largest of the 32 belongs to a third distinct id, hence
+        // is a lower bound of the CTA's third-largest bound.
+        float rs[N], t[N];
+        bounds(v_begin, p0, q0, rs, t);
+        float m = 0.f;
+#pragma unroll
+        for (int i = 0; i < N; ++i)
+            if (rs[i] > 0.f) m = fmaxf(m, __fdividef(rs[i], neg_log_uniform(t[i])));
+        unsigned bits = __float_as_uint(m);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {  // drop the lanes holding the largest and the second largest
+            const unsigned top_bits = __reduce_max_sync(0xFFFFFFFFu, bits);
+            const unsigned holders = __ballot_sync(0xFFFFFFFFu, bits == top_bits);
+            if (lane == __ffs(holders) - 1) bits = 0u;
+        }
+        floor_w = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, bits)) * 0.9999f;  // (the bounds above are not rounded up)
+        if (lane == 0) atomicMax(&sh.floor_bits, __float_as_uint(floor_w));
+    }
+#pragma unroll 1
+    for (int v0 = v_begin; v0 < v_end; v0 += 2 * kResidualThreads) {
+        fetch(v0 + 2 * kResidualThreads, p2, q2);
+        fetch(v0 + 3 * kResidualThreads, p3, q3);
+        floor_w = fmaxf(floor_w, __uint_as_float(*reinterpret_cast<volatile unsigned*>(&sh.floor_bits)));
+        float rs[2 * N], t[2 * N];
+        {
+            float (&rs0)[N] = *reinterpret_cast<float(*)[N]>(rs);
+            float (&t0)[N] = *reinterpret_cast<float(*)[N]>(t);
+            float (&rs1)[N] = *reinterpret_cast<float(*)[N]>(rs + N);
+            float (&t1)[N] = *reinterpret_cast<float(*)[N]>(t + N);
+            bounds(v0, p0, q0, rs0, t0);
+            bounds(v0 + kResidualThreads, p1, q1, rs1, t1);
+        }
+        unsigned qualify = 0u;
+#pragma unroll
+        for (int i = 0; i < 2 * N; ++i) qualify |= (rs[i] > floor_w * t[i]) ? (1u << i) : 0u;
+        if (__any_sync(0xFFFFFFFFu, qualify != 0u)) {
+#pragma unroll
+            for (int i = 0; i < 2 * N; ++i)
+                if (qualify & (1u << i))
+                    top = offer_bound(top, rs[i], t[i],
+                                      (v0 + (i / N) * kResidualThreads + static_cast<int>(threadIdx.x)) * N + (i % N));
+            // raise the floor: any lane's third-best bound is a lower bound of the CTA's third best
+            floor_w = fmaxf(floor_w, __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(top.w3))));
+            if (lane == 0) atomicMax(&sh.floor_bits, __float_as_uint(floor_w));  // shared without a barrier
+        }
+        p0 = p2;
+        q0 = q2;
+        p1 = p3;
+        q1 = q3;
     }
     // tail elements (beyond the last whole vector) belong to part 0
     if (part == 0) {
         for (int x = G.vec_elems + threadIdx.x; x < G.V; x += kResidualThreads) {
-            const float lp = load_logit<DT>(prow, x), lq = load_logit<DT>(qrow, x);
-            const float r = exp2_scaled<DT>(lp, P.c_hi, P.c_lo, kp) - exp2_scaled<DT>(lq, P.c_hi, P.c_lo, kq);
-            if (r > 0.f) {
+            const float ep = exp2_scaled<DT>(load_logit<DT>(prow, x), P.c_hi, P.c_lo, kp);
+            const float rsx = fmaf(ep, slack, ep - exp2_scaled<DT>(load_logit<DT>(qrow, x), P.c_hi, P.c_lo, kq));
+            if (rsx > 0.f) {
                 const uint4 w = rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(x + P.vocab_offset) >> 2));
-                const uint32_t word = (x & 3) == 0 ? w.x : (x & 3) == 1 ? w.y : (x & 3) == 2 ? w.z : w.w;
-                top.offer(__fdividef(r, neg_log_uniform(one_minus_uniform(word))), x);
+                top = offer_bound(top, rsx, one_minus_uniform(pick_word(w, x & 3)), x);
             }
         }
     }
 
-    // ---- CTA-wide best two
+    // ---- CTA-wide best three (warp results meet in shared memory, warp 0 folds them), then the
+    //      hand-over to the CTA that decides
     top.warp_merge();
-    __shared__ Top2 s_top[kResidualThreads / 32];
-    __shared__ int s_last;
-    __shared__ double s_score[kResidualThreads / 32];
-    __shared__ int s_x[kResidualThreads / 32];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) s_top[warp] = top;
+    if (lane == 0) sh.top[warp] = top;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        Top2 all = s_top[0];
-        for (int w = 1; w < kResidualThreads / 32; ++w) {
-            all.offer(s_top[w].w1, s_top[w].x1);
-            all.offer(s_top[w].w2, s_top[w].x2);
+    if (warp == 0) {
+        Top3 all;
+        all.clear();
+        if (lane < kResidualWarps) all = sh.top[lane];
+        all.warp_merge();
+        if (lane == 0) {
+            if constexpr (CLUSTER) {
+                // the window's CTAs form one cluster: candidates go to rank 0's shared memory
+                Candidate* out = cg::this_cluster().map_shared_rank(sh.cluster_cand, 0) + part * kCandidatesPerCta;
+                out[0].w = all.w1;
+                out[0].x = all.x1;
+                out[1].w = all.w2;
+                out[1].x = all.x2;
+                out[2].w = all.w3;
+                out[2].x = all.x3;
+            } else {
+                Candidate* out = P.candidates + (static_cast<int64_t>(b) * parts + part) * kCandidatesPerCta;
+                out[0].w = all.w1;
+                out[0].x = all.x1;
+                out[1].w = all.w2;
+                out[1].x = all.x2;
+                out[2].w = all.w3;
+                out[2].x = all.x3;
+                __threadfence();
+                const unsigned before = atomicAdd(&P.tasks[b].arrivals, 1u);
+                sh.last = (before == static_cast<unsigned>(parts) - 1u);
+            }
+            sh.exact = 0;
         }
-        Candidate* out = P.candidates + (static_cast<int64_t>(b) * parts + part) * 2;
-        out[0].w = all.w1;
-        out[0].x = all.x1;
-        out[1].w = all.w2;
-        out[1].x = all.x2;
+    }
+    if constexpr (CLUSTER) {
+        cg::this_cluster().sync();  // (every CTA of a window gets here or none does)
+        if (part != 0) return;
+    } else {
+        __syncthreads();
+        if (!sh.last) return;
         __threadfence();
-        const unsigned before = atomicAdd(&P.tasks[b].arrivals, 1u);
-        s_last = (before == static_cast<unsigned>(parts) - 1u);
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
 
-    // ---- the last CTA of the window decides, in double precision, among the
-    //      candidates whose binary32 weight is within 2^-9 of the best one
     const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
-    const volatile Candidate* cand = P.candidates + static_cast<int64_t>(b) * parts * 2;
-    float w = 0.f;
-    int x = 0x7FFFFFFF;
-    if (static_cast<int>(threadIdx.x) < 2 * parts) {
-        w = cand[threadIdx.x].w;
-        x = cand[threadIdx.x].x;
-    }
-    double wbest = w;
-    int dummy = 0;
-    block_argmax(wbest, dummy, s_score, s_x);
-    double score = -INFINITY;
-    int Z = 0x7FFFFFFF;
-    if (w > 0.f && static_cast<double>(w) >= wbest * (1.0 - 1.0 / 512.0)) {
-        score = exact_score<DT>(x, prow, qrow, c, task.kp, task.kq, ub, upos, P);
-        if (score > -INFINITY) Z = x;
-    }
-    block_argmax(score, Z, s_score, s_x);
+    const volatile Candidate* cand =
+        CLUSTER ? sh.cluster_cand : P.candidates + static_cast<int64_t>(b) * parts * kCandidatesPerCta;
+    const int ncand = parts * kCandidatesPerCta;
 
-    bool have_score = true;
-    if (!(score > -INFINITY)) {
-        // Nothing survived in binary32 (the residual mass is at rounding level or zero):
-        // go over the whole row in double precision.
-        score = -INFINITY;
-        Z = 0x7FFFFFFF;
-        for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
-            const double s = exact_score<DT>(xx, prow, qrow, c, task.kp, task.kq, ub, upos, P);
-            if (s > score) {  // increasing xx: the lowest index keeps a tie
-                score = s;
-                Z = xx;
+    if constexpr (!REPORT) {
+        // ---- one warp decides
+        if (warp == 0) {
+            Top3 all;
+            all.clear();
+            for (int j = lane; j < ncand; j += 32) all.offer(cand[j].w, cand[j].x);
+            all.warp_merge();
+            // lanes 0 and 1: the ids of the two largest bounds.  First in binary32 with the same bounds as
+            // the pass (a few hundred cycles); only when those do not separate them, in double precision.
+            const int xe = lane == 0 ? all.x1 : all.x2;
+            const float we = lane == 0 ? all.w1 : all.w2;
+            const bool have = lane < 2 && we > 0.f && xe >= 0 && xe < G.V;
+            float lpf = 0.f, lqf = 0.f, lb32 = -1.f, ub32 = 0.f;
+            uint32_t word = 0u;
+            if (have) {
+                lpf = load_logit<DT>(prow, xe);
+                lqf = load_logit<DT>(qrow, xe);
+                word = pick_word(rng.draw(P.keys, (kStreamResidual << 30) | (static_cast<uint32_t>(xe + P.vocab_offset) >> 2)),
+                                 xe & 3);
+                const float ep = exp2_scaled<DT>(lpf, P.c_hi, P.c_lo, kp);
+                const float r32 = ep - exp2_scaled<DT>(lqf, P.c_hi, P.c_lo, kq);
+                const float e32 = neg_log_uniform(one_minus_uniform(word));
+                ub32 = __fdividef(fmaf(ep, slack, r32), e32) * 1.00003f;
+                lb32 = __fdividef(fmaf(ep, -slack, r32), e32) * 0.99997f;
+            }
+            const float lb_a = __shfl_sync(0xFFFFFFFFu, lb32, 0), lb_b = __shfl_sync(0xFFFFFFFFu, lb32, 1);
+            const float ub_a = __shfl_sync(0xFFFFFFFFu, ub32, 0), ub_b = __shfl_sync(0xFFFFFFFFu, ub32, 1);
+            const bool first32 = lb_a >= lb_b;
+            const float lo32 = first32 ? lb_a : lb_b, hi32 = first32 ? ub_b : ub_a;
+            if (lo32 > 1e-37f && lo32 > hi32 && lo32 > all.w3) {  // (the same in every lane)
+                if (lane == (first32 ? 0 : 1)) {
+                    P.tokens[out_row] = xe;
+                    P.conf[out_row] = static_cast<float>(exp2(static_cast<double>(lpf) * c - kp_d));
+                }
+            } else {
+                double wn = -1.0, lo = -1.0, hi = 0.0, pi = 0.0;
+                if (have) {
+                    pi = exp2(static_cast<double>(lpf) * c - kp_d);
+                    const double r = pi - exp2(static_cast<double>(lqf) * c - kq_d);
+                    const double e = -log(static_cast<double>(uniform_from_word(word)));
+                    wn = r / e;
+                    lo = (r - 2.0 * kNormRelErr * pi) / e * (1.0 - 1e-12);
+                    hi = (r + 2.0 * kNormRelErr * pi) / e * (1.0 + 1e-12);
+                }
+                const double wn2 = __shfl_sync(0xFFFFFFFFu, wn, 1), lo2 = __shfl_sync(0xFFFFFFFFu, lo, 1);
+                const double hi2 = __shfl_sync(0xFFFFFFFFu, hi, 1), pi2 = __shfl_sync(0xFFFFFFFFu, pi, 1);
+                if (lane == 0) {
+                    const bool first = wn >= wn2;
+                    const double lo_w = first ? lo : lo2, hi_o = first ? hi2 : hi;
+                    if (lo_w > 1e-300 && lo_w > hi_o && lo_w > static_cast<double>(all.w3)) {
+                        P.tokens[out_row] = first ? all.x1 : all.x2;
+                        P.conf[out_row] = static_cast<float>(first ? pi : pi2);
+                    } else {
+                        sh.exact = 1;
+                        // a lower bound of the largest true weight, rounded down, for the double-precision pass
+                        const double lb = fmax(fmax(lo, lo2), 0.0);
+                        sh.exact_floor = lb > 1e-30 ? __double2float_rd(lb) * (1.0f - 1e-6f) : 0.f;
+                    }
+                }
             }
         }
-        block_argmax(score, Z, s_score, s_x);
+        __syncthreads();
+        if (!sh.exact) return;
+        int Z;
+        double piZ;
+        exact_row_draw<DT>(P, prow, qrow, ub, upos, kp_d, kq_d, slack, sh.exact_floor, sh, Z, piZ);
+        if (threadIdx.x == 0) {
+            if (Z < 0 || Z >= G.V) {  // no finite target logit: the scan has reported such a row already
+                P.tokens[out_row] = -1;
+                P.conf[out_row] = -1.f;
+                report(P.status, FEF_ERR_NONFINITE);
+            } else {
+                P.tokens[out_row] = Z;
+                P.conf[out_row] = static_cast<float>(piZ);
+            }
+        }
+    } else {
+        // ---- this rank's best id by its score under the shared normalisers: candidates whose bound
+        //      is within a band of the largest are scored in double precision
+        // (at most kMaxResidualCtas * kCandidatesPerCta = 2 * kResidualThreads candidates: two per thread)
+        float w[2] = {0.f, 0.f};
+        int x[2] = {0x7FFFFFFF, 0x7FFFFFFF};
+        double wbest = 0.0;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int j = static_cast<int>(threadIdx.x) + k * kResidualThreads;
+            if (j < ncand) {
+                w[k] = cand[j].w;
+                x[k] = cand[j].x;
+            }
+            wbest = fmax(wbest, static_cast<double>(w[k]));
+        }
+        int dummy = 0;
+        block_argmax(wbest, dummy, sh);
+        const double band = fmax(1.0 / 512.0, 64.0 * static_cast<double>(slack));
+        double score = -INFINITY;
+        int Z = 0x7FFFFFFF;
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+            if (w[k] > 0.f && static_cast<double>(w[k]) >= wbest * (1.0 - band)) {
+                const double sc = exact_score<DT>(x[k], prow, qrow, c, kp_d, kq_d, ub, upos, P);
+                if (sc > score || (sc == score && sc > -INFINITY && x[k] < Z)) {
+                    score = sc;
+                    Z = x[k];
+                }
+            }
+        block_argmax(score, Z, sh);
+        bool have_score = true;
         if (!(score > -INFINITY)) {
-            // [pi - rho]_+ is identically zero: commit arg-max of pi (= arg-max of the target logits)
-            have_score = false;
+            // nothing with a positive residual among the candidates: go over the slice in double precision
             score = -INFINITY;
             Z = 0x7FFFFFFF;
             for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
-                const double l = load_logit<DT>(prow, xx);
-                if (l > score) {
-                    score = l;
+                const double s = exact_score<DT>(xx, prow, qrow, c, kp_d, kq_d, ub, upos, P);
+                if (s > score) {  // increasing xx: the lowest index keeps a tie
+                    score = s;
                     Z = xx;
                 }
             }
-            block_argmax(score, Z, s_score, s_x);
+            block_argmax(score, Z, sh);
+            if (!(score > -INFINITY)) {
+                // [pi - rho]_+ is zero on the slice: report the arg-max of the target logits
+                have_score = false;
+                score = -INFINITY;
+                Z = 0x7FFFFFFF;
+                for (int xx = threadIdx.x; xx < G.V; xx += kResidualThreads) {
+                    const double l = load_logit<DT>(prow, xx);
+                    if (l > score) {
+                        score = l;
+                        Z = xx;
+                    }
+                }
+                block_argmax(score, Z, sh);
+            }
+        }
+        if (threadIdx.x == 0) {
+            const bool none = Z < 0 || Z >= G.V;  // the slice holds no finite target logit
+            VpCandidate out;
+            out.score = (have_score && !none) ? score : -INFINITY;
+            out.lp = none ? -INFINITY : load_logit<DT>(prow, Z);
+            out.index = none ? 0x7FFFFFFF : Z + P.vocab_offset;
+            P.vp_out[b] = out;
+        }
+    }
+}
+
+// Vocabulary-parallel mode: the residual draw over this rank's slice for the windows whose task
+// (written by vp_accept_kernel) names a rejected position.
+template <int DT>
+__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual_kernel(const __grid_constant__ VerifyParams P) {
+    __shared__ ResidualShared sh;
+    cudaGridDependencySynchronize();
+    const int b = blockIdx.y;
+    const ResidualTask task = P.tasks[b];
+    if (task.pos < 0) return;  // uniform over the CTA
+    if (threadIdx.x == 0) sh.floor_bits = 0u;
+    __syncthreads();
+    const int64_t row = static_cast<int64_t>(b) * P.geo.K + task.pos;
+    residual_draw<DT, true, false>(P, b, task.pos, task.kp, task.kq, P.target + row * P.geo.ld_bytes,
+                            P.draft + row * P.geo.ld_bytes, row, blockIdx.x, gridDim.x, sh);
+}
+
+// ================================================================= tail ====
+// Sampling mode, everything after the streaming kernel in one launch (Algorithm 2, "for m = 1..b"
+// from the acceptance test on): grid (parts, B).  Every CTA of window b repeats the window's
+// acceptance tests from the partials (a few hundred operations per position, the same in every
+// CTA, so all agree on the first rejection without talking to each other); part 0 writes the accepted
+// tokens and confidences; then the CTAs share the residual draw of the rejected row.
+struct TailShared {
+    double kp[FEF_MAX_K], kq[FEF_MAX_K];
+    float conf[FEF_MAX_K];
+    int tok[FEF_MAX_K];
+    unsigned rejected[FEF_MAX_K / 32];
+    int err;
+};
+
+// One position's acceptance test from its folded normalisers.  Returns 0 or a data error.
+__device__ __forceinline__ int accept_test(const VerifyParams& P, int b, int i, int x, double lpx, double lqx,
+                                           const RowNorm& np, const RowNorm& nq, double c, TailShared& ts) {
+    const Geometry& G = P.geo;
+    if (x < 0 || x >= G.V) return FEF_ERR_TOKEN_RANGE;
+    if (np.bad || nq.bad) return FEF_ERR_NONFINITE;
+    const double kp = np.M + log2(np.S);
+    const double kq = nq.M + log2(nq.S);
+    const double l2pi = lpx * c - kp;  // log2 pi(x)
+    bool accept;
+    if (lqx == -INFINITY) {
+        accept = lpx > -INFINITY;  // rho(x) = 0: accept iff pi(x) > 0
+    } else {
+        const double ratio = exp2(l2pi - (lqx * c - kq));
+        const uint4 rnd = philox4x32_10(
+            make_uint4(kStreamAccept << 30, static_cast<uint32_t>(b), static_cast<uint32_t>(i), step_of(P)),
+            make_uint2(static_cast<uint32_t>(P.seed), static_cast<uint32_t>(P.seed >> 32)));
+        accept = static_cast<double>(uniform_from_word(rnd.x)) <= fmin(1.0, ratio);
+    }
+    ts.kp[i] = kp;
+    ts.kq[i] = kq;
+    ts.conf[i] = static_cast<float>(exp2(l2pi));
+    ts.tok[i] = x;
+    if (!accept) atomicOr(&ts.rejected[i >> 5], 1u << (i & 31));
+    return 0;
+}
+
+template <int DT, bool CLUSTER>
+__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_kernel(const __grid_constant__ VerifyParams P) {
+    const Geometry& G = P.geo;
+    __shared__ TailShared ts;
+    __shared__ ResidualShared sh;
+    const int b = blockIdx.y, part = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    // few rows, many partials per row: a warp per position shares the fold; otherwise a thread per position
+    const bool wide = G.claims_per_unit >= 4;
+
+    // what does not depend on the streaming kernel is fetched before waiting for it: the draft token
+    // of "my" position and the two logits at it.  Thread form: position threadIdx.x.  Warp form: lane j
+    // of warp w holds position w + j * kResidualWarps.
+    const int my = wide ? (lane < FEF_MAX_K / kResidualWarps ? warp + lane * kResidualWarps : FEF_MAX_K)
+                        : static_cast<int>(threadIdx.x);
+    int x = -1;
+    double lpx = 0.0, lqx = 0.0;
+    if (my < n) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + my;
+        x = __ldg(P.draft_tokens + row);
+        if (x >= 0 && x < G.V) {
+            lpx = load_logit<DT>(P.target + row * G.ld_bytes, x);
+            lqx = load_logit<DT>(P.draft + row * G.ld_bytes, x);
         }
     }
     if (threadIdx.x == 0) {
-        // Z stays "none" when the row (vocabulary-parallel mode: this rank's slice of it) holds no finite
-        // target logit; a whole row like that has been reported by the scan already
-        const bool none = Z < 0 || Z >= G.V;
-        const float lp = none ? -INFINITY : load_logit<DT>(prow, Z);
-        if (none && !P.vp_out) {
-            P.tokens[row] = -1;
-            P.conf[row] = -1.f;
-            report(P.status, FEF_ERR_NONFINITE);
-        } else if (P.vp_out) {  // vocabulary-parallel: this rank's best; the ranks' reports are compared afterwards
-            VpCandidate out;
-            out.score = (have_score && !none) ? score : -INFINITY;
-            out.lp = lp;
-            out.index = none ? 0x7FFFFFFF : Z + P.vocab_offset;
-            P.vp_out[b] = out;
-        } else {
-            P.tokens[row] = Z;
-            P.conf[row] = static_cast<float>(exp2(static_cast<double>(lp) * c - task.kp));
+        ts.rejected[0] = ts.rejected[1] = 0u;
+        ts.err = 0;
+        sh.floor_bits = 0u;
+    }
+    __syncthreads();
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+
+    if (!wide) {
+        if (my < n) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + my;
+            const RowNorm np = fold_unit<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P);
+            RowNorm nq;
+            if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
+                nq.M = P.draft_norm[row];
+                nq.S = 1.0;
+                nq.bad = !(fabs(nq.M) < INFINITY);
+            } else {
+                nq = fold_unit<DT, false>(2 * row + 1, P.draft + row * G.ld_bytes, c, P);
+            }
+            const int e = accept_test(P, b, my, x, lpx, lqx, np, nq, c, ts);
+            if (e) atomicMax(&ts.err, e);
+        }
+    } else {
+        for (int j = 0; j < FEF_MAX_K / kResidualWarps; ++j) {
+            const int i = warp + j * kResidualWarps;
+            if (i >= n) break;  // uniform over the warp
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
+            const RowNorm np = fold_unit_warp<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P, lane);
+            RowNorm nq;
+            if (P.draft_norm) {
+                nq.M = P.draft_norm[row];
+                nq.S = 1.0;
+                nq.bad = !(fabs(nq.M) < INFINITY);
+            } else {
+                nq = fold_unit_warp<DT, false>(2 * row + 1, P.draft + row * G.ld_bytes, c, P, lane);
+            }
+            const int xi = __shfl_sync(0xFFFFFFFFu, x, j);
+            const double lpi = __shfl_sync(0xFFFFFFFFu, lpx, j), lqi = __shfl_sync(0xFFFFFFFFu, lqx, j);
+            if (lane == 0) {
+                const int e = accept_test(P, b, i, xi, lpi, lqi, np, nq, c, ts);
+                if (e) atomicMax(&ts.err, e);
+            }
         }
     }
+    __syncthreads();
+
+    const int err = ts.err;
+    int a = n;
+    if (ts.rejected[0])
+        a = __ffs(ts.rejected[0]) - 1;
+    else if (ts.rejected[1])
+        a = 32 + __ffs(ts.rejected[1]) - 1;
+
+    if (part == 0) {
+        for (int i = threadIdx.x; i < G.K; i += kResidualThreads) {
+            const int64_t row = static_cast<int64_t>(b) * G.K + i;
+            const bool keep = !err && i < a;
+            P.tokens[row] = keep ? ts.tok[i] : -1;
+            P.conf[row] = keep ? ts.conf[i] : -1.f;
+        }
+        if (threadIdx.x == 0) {
+            P.accept_len[b] = err ? -1 : a;
+            if (err) report(P.status, err);
+        }
+    }
+    if (err || a >= n) return;  // uniform over the CTA (and over the window's CTAs)
+    const int64_t row = static_cast<int64_t>(b) * G.K + a;
+    residual_draw<DT, false, CLUSTER>(P, b, a, ts.kp[a], ts.kq[a], P.target + row * G.ld_bytes, P.draft + row * G.ld_bytes, row, part,
+                             static_cast<int>(gridDim.x), sh);
 }
 
 // =================================================== vocabulary-parallel ====
@@ -1404,7 +1762,7 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool ta
     // residual kernel: CTAs per rejected row, each thread up to kResidualBatch vector pairs
     // (fewer when few windows would leave SMs idle)
     const int nvec = G.vec_bytes / 16;
-    int per_thread = kResidualBatch;
+    int per_thread = 4;
     while (per_thread > 1 &&
            static_cast<int64_t>(B) * ((nvec + kResidualThreads * per_thread - 1) / (kResidualThreads * per_thread)) < 2 * sm_count)
         per_thread >>= 1;
@@ -1433,7 +1791,7 @@ static WorkspaceLayout layout_of(const Geometry& G) {
     L.partials = L.zero_bytes;
     L.tasks = L.partials + round256(static_cast<size_t>(G.num_claims) * sizeof(Partial));
     L.candidates = L.tasks + round256(static_cast<size_t>(G.B) * sizeof(ResidualTask));
-    L.total = L.candidates + round256(static_cast<size_t>(G.B) * kMaxResidualCtas * 2 * sizeof(Candidate));
+    L.total = L.candidates + round256(static_cast<size_t>(G.B) * kMaxResidualCtas * kCandidatesPerCta * sizeof(Candidate));
     return L;
 }
 
@@ -1455,12 +1813,33 @@ static cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 blo
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
+// The same with the CTAs of a grid row (blockIdx.y) grouped into one thread-block cluster.
+template <typename... Args>
+static cudaError_t launch_dependent_cluster(int cluster_x, void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem,
+                                            cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(cluster_x);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
 
 static void mark(void* const* events, int which, cudaStream_t stream) {
     if (events && events[which]) cudaEventRecord(static_cast<cudaEvent_t>(events[which]), stream);
 }
 
-// events (may be null): [0] before the streaming kernel, [1] after it, [2] after the scan, [3] at the end
+// events (may be null): [0] before the streaming kernel, [1] after it, [2] and [3] after the kernel
+// that follows it (sampling mode: acceptance tests and residual draw in one launch; greedy mode: the scan)
 template <int DT, bool GREEDY>
 static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t stream, void* const* events) {
     const Geometry& G = P.geo;
@@ -1472,37 +1851,43 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         g_attr_done[dev][which] = true;
     }
     cudaError_t e;
-    if (G.warp_per_row) {
-        if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
-        mark(events, 0, stream);
-        e = launch_dependent(rows_kernel<DT, GREEDY>, dim3(G.grid), dim3(kRowsWarps * 32), 0, stream, P);
-        if (e != cudaSuccess) return e;
-    } else if (events) {
+    if (events) {
         // timing marks asked for: clear with memset nodes and launch the streaming kernel the
         // ordinary way, so that the first two marks bracket that kernel alone
         if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
         if ((e = cudaMemsetAsync(P.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return e;
+        if ((e = cudaMemsetAsync(P.tasks, 0, sizeof(ResidualTask) * G.B, stream)) != cudaSuccess) return e;
         mark(events, 0, stream);
-        stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, kSmemBytes, stream>>>(P);
+        if (G.warp_per_row)
+            rows_kernel<DT, GREEDY><<<G.grid, kRowsWarps * 32, 0, stream>>>(P);
+        else
+            stream_kernel<DT, GREEDY><<<G.grid, kStreamThreads, kSmemBytes, stream>>>(P);
     } else {
-        e = launch_dependent(begin_call_kernel, dim3(1), dim3(32), 0, stream, P.ctl, P.status);
+        e = launch_dependent(begin_call_kernel, dim3(1), dim3(kBeginThreads), 0, stream, P.ctl, P.tasks, G.B, P.status);
         if (e != cudaSuccess) return e;
-        e = launch_dependent(stream_kernel<DT, GREEDY>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
+        if (G.warp_per_row)
+            e = launch_dependent(rows_kernel<DT, GREEDY>, dim3(G.grid), dim3(kRowsWarps * 32), 0, stream, P);
+        else
+            e = launch_dependent(stream_kernel<DT, GREEDY>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
         if (e != cudaSuccess) return e;
     }
     mark(events, 1, stream);
-    if (G.claims_per_unit >= 4)  // few rows, many partials per row: one warp per position
-        e = launch_dependent(scan_rows_kernel<DT, GREEDY>, dim3(G.B),
-                             dim3(32 * (G.K < kScanMaxWarps ? G.K : kScanMaxWarps)), 0, stream, P);
-    else
-        e = launch_dependent(scan_kernel<DT, GREEDY>, dim3((G.B + kScanWarps - 1) / kScanWarps), dim3(kScanWarps * 32),
-                             0, stream, P);
+    if constexpr (GREEDY) {
+        if (G.claims_per_unit >= 4)  // few rows, many partials per row: one warp per position
+            e = launch_dependent(scan_rows_kernel<DT>, dim3(G.B), dim3(32 * (G.K < kScanMaxWarps ? G.K : kScanMaxWarps)), 0,
+                                 stream, P);
+        else
+            e = launch_dependent(scan_kernel<DT>, dim3((G.B + kScanWarps - 1) / kScanWarps), dim3(kScanWarps * 32), 0,
+                                 stream, P);
+    } else {
+        if (G.residual_ctas <= kMaxClusterCtas)
+            e = launch_dependent_cluster(G.residual_ctas, tail_kernel<DT, true>, dim3(G.residual_ctas, G.B),
+                                         dim3(kResidualThreads), 0, stream, P);
+        else
+            e = launch_dependent(tail_kernel<DT, false>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
+    }
     if (e != cudaSuccess) return e;
     mark(events, 2, stream);
-    if (!GREEDY) {
-        e = launch_dependent(residual_kernel<DT>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
-        if (e != cudaSuccess) return e;
-    }
     mark(events, 3, stream);
     return cudaGetLastError();
 }
@@ -1581,6 +1966,7 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
         P.c_lo = 0.f;
     }
     P.c_hi = c_hi;
+    P.c_exact = c;
     if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
 
     P.target = static_cast<const char*>(target_logits);
@@ -1695,6 +2081,7 @@ static fef_status vp_setup(const void* draft_slice, const void* target_slice, co
         if (!(P.c_lo > 0.f)) return FEF_ERR_INVALID_ARG;
     }
     P.c_hi = c_hi;
+    P.c_exact = c;
     if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
     P.target = static_cast<const char*>(target_slice);
     P.draft = static_cast<const char*>(draft_slice);
@@ -1732,7 +2119,8 @@ static cudaError_t vp_launch_stats(const fef::VerifyParams& P, int dev, double* 
         if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
         e = launch_dependent(rows_kernel<DT, false>, dim3(G.grid), dim3(kRowsWarps * 32), 0, stream, P);
     } else {
-        e = launch_dependent(begin_call_kernel, dim3(1), dim3(32), 0, stream, P.ctl, P.status);
+        e = launch_dependent(begin_call_kernel, dim3(1), dim3(kBeginThreads), 0, stream, P.ctl,
+                             static_cast<ResidualTask*>(nullptr), 0, P.status);
         if (e != cudaSuccess) return e;
         e = launch_dependent(stream_kernel<DT, false>, dim3(G.grid), dim3(kStreamThreads), kSmemBytes, stream, P);
     }

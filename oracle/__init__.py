@@ -20,7 +20,7 @@ _HDR = os.path.join(_HERE, "fef_oracle.h")
 _LIB = os.path.join(_HERE, "libfef_oracle.so")
 
 OK, ERR_INVALID_ARG, ERR_DTYPE, ERR_NONFINITE, ERR_TOKEN_RANGE = 0, 1, 2, 7, 8
-F32, BF16 = 0, 1
+F32, BF16, F64 = 0, 1, 2
 
 _lock = threading.Lock()
 _lib = None
@@ -83,8 +83,12 @@ def _logits_as_numpy(x):
             return x.view(torch.int16).numpy().view(np.uint16), BF16
         if x.dtype == torch.float32:
             return x.numpy(), F32
+        if x.dtype == torch.float64:
+            return x.numpy(), F64
         raise ValueError("logits must be float32 or bfloat16")
     x = np.ascontiguousarray(x)
+    if x.dtype == np.float64:
+        return x, F64
     if x.dtype == np.float32:
         return x, F32
     if x.dtype == np.uint16:  # raw bfloat16 bit patterns

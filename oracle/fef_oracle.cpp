@@ -32,6 +32,9 @@ const double kInf = std::numeric_limits<double>::infinity();
 
 // ---------------------------------------------------------------- logits ----
 double load_logit(const void* base, int64_t index, int dtype) {
+    if (dtype == FEFO_F64) {
+        return static_cast<const double*>(base)[index];
+    }
     if (dtype == FEFO_F32) {
         return (double)static_cast<const float*>(base)[index];
     }
@@ -339,12 +342,12 @@ int fef_oracle_spec_verify(const void* draft_logits, const void* target_logits,
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
         return FEFO_ERR_INVALID_ARG;
     if (B < 1 || K < 1 || V < 1 || ld < V || !(temperature >= 0.0f)) return FEFO_ERR_INVALID_ARG;
-    if (dtype != FEFO_F32 && dtype != FEFO_BF16) return FEFO_ERR_DTYPE;
+    if (dtype != FEFO_F32 && dtype != FEFO_BF16 && dtype != FEFO_F64) return FEFO_ERR_DTYPE;
     if (row_len)
         for (int b = 0; b < B; ++b)
             if (row_len[b] < 0 || row_len[b] > K) return FEFO_ERR_INVALID_ARG;
 
-    const int64_t elem = (dtype == FEFO_F32) ? 4 : 2;
+    const int64_t elem = (dtype == FEFO_F64) ? 8 : (dtype == FEFO_F32) ? 4 : 2;
     int worst = FEFO_OK;
     for (int b = 0; b < B; ++b) {
         const int64_t window = (int64_t)b * K;

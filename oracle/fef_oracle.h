@@ -41,8 +41,9 @@ enum {
     FEFO_ERR_TOKEN_RANGE = 8
 };
 
-/* logit storage types */
-enum { FEFO_F32 = 0, FEFO_BF16 = 1 };
+/* logit storage types (FEFO_F64: fef_oracle_spec_verify only; logits that come out of a
+ * double-precision matrix product, see oracle/lmhead.py) */
+enum { FEFO_F32 = 0, FEFO_BF16 = 1, FEFO_F64 = 2 };
 
 /* Philox4x32-10 block function: out[4] = philox(ctr[4], key[2]). */
 void fef_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
@@ -64,7 +65,7 @@ int fef_oracle_row_laws(const void* p_logits, const void* q_logits, int V, int d
 
 /* One verification call over B independent windows of K positions
  * (Algorithm 2, the loop "for m = 1..b").
- *   draft_logits, target_logits : [B, K, ld] (ld >= V), dtype F32 or BF16
+ *   draft_logits, target_logits : [B, K, ld] (ld >= V), dtype F32, BF16 or F64
  *   draft_tokens                : [B, K]
  *   row_len                     : [B] number of valid drafts (0..K), or NULL = K
  *   temperature                 : > 0 sampling; == 0 greedy (see the notes at the top of

@@ -681,3 +681,57 @@ def test_loop_toy_run_resolves_everything_and_remasks_the_lowest_confidences():
         assert sorted(pos[b].tolist()) == sorted(np.argsort(conf[b], kind="stable")[:k].tolist())
     oloop.remask(tokens, conf, in_step, pos, cnt)
     assert ((tokens == oloop.MASK).sum(axis=1) == k).all()
+
+
+# ------------------------------------------------ logits from hidden states ----
+def test_lmhead_product_equals_exact_integer_arithmetic():
+    """Small integer-valued bfloat16 inputs: every product and sum is an integer below 2^53, so the
+    double-precision product must equal Python's exact integers."""
+    from oracle import lmhead
+
+    rng = np.random.default_rng(5)
+    R, d, V = 5, 37, 11
+    H = rng.integers(-9, 10, size=(R, d))
+    W = rng.integers(-7, 8, size=(V, d))
+    got = lmhead.lmhead_logits(torch.tensor(H, dtype=torch.bfloat16), torch.tensor(W, dtype=torch.bfloat16))
+    want = [[sum(int(H[r, k]) * int(W[v, k]) for k in range(d)) for v in range(V)] for r in range(R)]
+    assert got.shape == (R, V) and (got == np.array(want, dtype=np.float64)).all()
+    # weight = rows of the identity: the logits are the hidden states themselves (operand order, no transpose slip)
+    Hf = torch.randn(4, 6).to(torch.bfloat16)
+    eye = torch.eye(6, dtype=torch.bfloat16)[:5]
+    assert (lmhead.lmhead_logits(Hf, eye) == Hf.double().numpy()[:, :5]).all()
+
+
+def test_float64_logit_storage_equals_the_float32_path_on_shared_values():
+    """Logits that float32 holds exactly give the same verification whether stored as float32 or float64."""
+    from paper_2605_14305_b200 import synth
+
+    w = synth.TINY.with_(B=3, K=4, V=200)
+    q, p, tok = synth.make_call(w, seed=12)
+    a = oracle.spec_verify(q, p, tok, 0.9, 3, 4)
+    b = oracle.spec_verify(q.double().numpy(), p.double().numpy(), tok, 0.9, 3, 4)
+    for key in ("accept_len", "tokens", "conf", "accept_margin", "gumbel_gap"):
+        assert (a[key] == b[key]).all(), key
+
+
+def test_lmhead_spec_verify_is_the_verification_of_its_own_logits():
+    from oracle import lmhead
+
+    g = torch.Generator().manual_seed(2)
+    B, K, d, V = 2, 3, 16, 50
+    Hq = torch.randn((B * K, d), generator=g).to(torch.bfloat16)
+    Hp = (Hq.float() + 0.3 * torch.randn((B * K, d), generator=g)).to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=g) * 0.5).to(torch.bfloat16)
+    tok = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    out = lmhead.lmhead_spec_verify(Hq, Hp, W, tok, B, K, 1.0, 9, 1)
+    again = oracle.spec_verify(out["draft_logits"], out["target_logits"], tok, 1.0, 9, 1)
+    assert (out["tokens"] == again["tokens"]).all() and (out["conf"] == again["conf"]).all()
+    # a common shift of one window's hidden states along a direction orthogonal to every weight row
+    # leaves the logits, hence the result, unchanged
+    Wn = W.clone()
+    Wn[:, 0] = 0
+    Hs = Hp.clone()
+    Hs[:, 0] += 4.0
+    o1 = lmhead.lmhead_spec_verify(Hq, Hp, Wn, tok, B, K, 1.0, 9, 1)
+    o2 = lmhead.lmhead_spec_verify(Hq, Hs, Wn, tok, B, K, 1.0, 9, 1)
+    assert (o1["tokens"] == o2["tokens"]).all() and (o1["conf"] == o2["conf"]).all()

@@ -369,7 +369,8 @@ def run_native(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": _config_dict(w, {"parallelism": "replicas x%d (windows are independent; no collective)" % world}),
+        "dtype": "f32", "data": "synthetic", "config": _config_dict(w),
+        "parallelism": "replicas x%d (windows are independent; no collective)" % world,
         "impl": "native",
         "hbm_gbs_whole_step": call_bytes / (elapsed_ms / steps * 1e-3) / 1e9,
         "frac_of_8TBs_whole_step": call_bytes / (elapsed_ms / steps * 1e-3) / 8e12,
@@ -426,7 +427,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": elapsed / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": _config_dict(w, {"parallelism": "one host thread"}),
+        "config": _config_dict(w), "parallelism": "one host thread",
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                          "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -493,6 +494,12 @@ def main():
     ap.add_argument("--no-call-events", action="store_true")
     ap.add_argument("--loop-sweep", action="store_true", help="time the full decoding loop at the sweep points instead")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.loop_sweep:
+        # started by hand for several GPUs: become one rank per GPU (the same launch the driver uses)
+        port = str(29500 + os.getpid() % 2000)
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node",
+                                   str(args.gpus), "--master-addr", "127.0.0.1", "--master-port", port,
+                                   os.path.abspath(__file__)] + sys.argv[1:])
     if args.loop_sweep:
         run_loop_sweep(args)
     elif args.impl == "reference":

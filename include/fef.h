@@ -395,6 +395,40 @@ fef_status fef_vp_finish(const void* candidates_all, int ranks, const void* task
                          int B, int K, fef_dtype dt, float temperature,
                          int32_t* tokens, float* conf, void* cuda_stream);
 
+/*
+ * Verification straight from hidden states (Section 3.2: the draft law rho^i and the target law pi^i
+ * are outputs of the model, i.e. softmax of hidden state x output-layer weight; Algorithm 2's loop
+ * over the window's positions and the residual law defined before it, as in fef_spec_verify).
+ *
+ *   logits^p[b,i,v] = sum_k target_hidden[b*K+i, k] * weight[v, k]      (and ^q with draft_hidden),
+ * accumulated in binary32 on the tensor cores from the bfloat16 inputs and never rounded to
+ * bfloat16 or written out: the product's epilogue keeps, per row and vocabulary chunk, the softmax
+ * partial sums and the logit at the draft token.  From there the call is fef_spec_verify on those
+ * binary32 logits: same acceptance rule, same random numbers (Philox counters as documented there),
+ * same outputs and sentinels.  The residual draw recomputes the logits of the rejected positions
+ * (2 B rows) with a second, small product.  Sampling mode only (temperature > 0).
+ *
+ *   draft_hidden, target_hidden  device, [B*K, d] bfloat16 row-major, 16-byte aligned
+ *   weight                       device, [V, d] bfloat16 row-major (the output layer), 16-byte aligned
+ *   d                            hidden width, a multiple of 8
+ *   workspace                    device scratch of fef_lmhead_verify_workspace_bytes(B, K, V, d) bytes
+ *                                (it holds, among others, the 2 B rows of binary32 logits), 256-byte aligned
+ * Everything else as in fef_spec_verify.  Asynchronous on `cuda_stream`; five kernels.
+ *
+ * fef_lmhead_logits writes the same binary32 logits for arbitrary rows, logits[r, v] for r < rows
+ * (ldo >= V elements per row, a multiple of 4): what the verification above sees, for inspection.
+ */
+size_t fef_lmhead_verify_workspace_bytes(int B, int K, int V, int d);
+fef_status fef_lmhead_verify(const void* draft_hidden, const void* target_hidden, const void* weight,
+                             const int32_t* draft_tokens, const int32_t* row_len,
+                             int B, int K, int V, int d,
+                             float temperature, uint64_t seed, uint32_t step,
+                             int32_t* accept_len, int32_t* tokens, float* conf,
+                             void* workspace, size_t workspace_bytes,
+                             int32_t* device_status, void* cuda_stream);
+fef_status fef_lmhead_logits(const void* hidden, const void* weight, int rows, int V, int d,
+                             float* logits, int64_t ldo, int32_t* device_status, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -57,11 +57,15 @@ LEDGER = ParityReport()
 
 
 def compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int = 0,
-                   ledger: bool = True) -> ParityReport:
+                   ledger: bool = True, margin: float = MARGIN, conf_rtol: float = CONF_RTOL) -> ParityReport:
     """``got_*``: arrays of the implementation under test for the same windows as ``ref``
     (the dict returned by ``oracle.spec_verify``).  The result is also added to ``LEDGER``
-    unless ``ledger`` is false."""
-    rep = _compare_verify(got_accept_len, got_tokens, got_conf, ref, batch_offset)
+    unless ``ledger`` is false.  ``margin`` / ``conf_rtol``: other bars than the standard ones, for
+    an implementation whose inputs themselves carry a stated error (logits from a binary32 product
+    against the oracle's double-precision product); such comparisons stay out of the ledger."""
+    rep = _compare_verify(got_accept_len, got_tokens, got_conf, ref, batch_offset, margin, conf_rtol)
+    if margin != MARGIN or conf_rtol != CONF_RTOL:
+        ledger = False
     if ledger:
         LEDGER.windows += rep.windows
         LEDGER.draws += rep.draws
@@ -72,7 +76,8 @@ def compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset
     return rep
 
 
-def _compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int) -> ParityReport:
+def _compare_verify(got_accept_len, got_tokens, got_conf, ref: dict, batch_offset: int, MARGIN: float,
+                    CONF_RTOL: float) -> ParityReport:
     ga = np.asarray(got_accept_len)
     gt = np.asarray(got_tokens)
     gc = np.asarray(got_conf, dtype=np.float64)

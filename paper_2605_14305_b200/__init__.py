@@ -8,6 +8,7 @@ compute function without the built library or without a CUDA device raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from typing import NamedTuple, Optional
@@ -28,7 +29,8 @@ EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_ver
            "fef_draft_sample_workspace_bytes", "fef_draft_sample", "fef_spec_verify_with_draft_norm",
            "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask",
            "fef_draft_sample_at_round", "fef_spec_verify_at_round", "fef_loop_advance_round",
-           "fef_vp_task_bytes", "fef_vp_local_stats", "fef_vp_accept", "fef_vp_local_residual", "fef_vp_finish")
+           "fef_vp_task_bytes", "fef_vp_local_stats", "fef_vp_accept", "fef_vp_local_residual", "fef_vp_finish",
+           "fef_lmhead_verify_workspace_bytes", "fef_lmhead_verify", "fef_lmhead_logits")
 
 _lib = None
 
@@ -98,6 +100,12 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_loop_remask.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
     for fn in (L.fef_loop_next_window, L.fef_loop_verification_inputs, L.fef_loop_commit, L.fef_loop_remask):
         fn.restype = i32
+    L.fef_lmhead_verify_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.fef_lmhead_verify_workspace_bytes.restype = sz
+    L.fef_lmhead_verify.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp, sz, vp, vp]
+    L.fef_lmhead_verify.restype = i32
+    L.fef_lmhead_logits.argtypes = [vp, vp, i32, i32, i32, vp, i64, vp, vp]
+    L.fef_lmhead_logits.restype = i32
     L.fef_remask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.fef_remask_select.restype = i32
     L.fef_remask_select_host_arena_bytes.argtypes = [i32, i32, i32]
@@ -126,6 +134,19 @@ def _require_cuda(*tensors):
     for t in tensors:
         if t is not None and t.device.type != "cuda":
             raise ValueError("all tensors must live on a CUDA device")
+
+
+@contextlib.contextmanager
+def _on(device, stream):
+    """``device`` current and, when a stream is given, that stream current as well: what a wrapper
+    allocates inside (outputs, scratch) then belongs to the stream its kernels run on, so the
+    caching allocator cannot hand the memory to someone else while those kernels still use it."""
+    with torch.cuda.device(device):
+        if stream is None:
+            yield
+        else:
+            with torch.cuda.stream(stream):
+                yield
 
 
 def _stream_ptr(stream) -> int:
@@ -177,7 +198,7 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
     V = ld if V is None else int(V)
     code = _dtype_code(draft_logits)
     dev = draft_logits.device
-    with torch.cuda.device(dev):
+    with _on(dev, stream):
         if out is None:
             out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
                                torch.empty((B, K), dtype=torch.int32, device=dev),
@@ -241,7 +262,7 @@ def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, 
     V = ld if V is None else int(V)
     code = _dtype_code(draft_logits)
     dev = draft_logits.device
-    with torch.cuda.device(dev):
+    with _on(dev, stream):
         if out is None:
             out = DraftResult(torch.empty((B, K), dtype=torch.int32, device=dev),
                               torch.empty((B, K), dtype=torch.float64, device=dev),
@@ -278,7 +299,7 @@ def fef_loop_next_window(tokens: torch.Tensor, K: int, stream=None):
     _i32_cuda(tokens, "fef_loop_next_window")
     B, L = tokens.shape
     dev = tokens.device
-    with torch.cuda.device(dev):
+    with _on(dev, stream):
         window = torch.empty((B, K), dtype=torch.int32, device=dev)
         row_len = torch.empty(B, dtype=torch.int32, device=dev)
         unresolved = torch.empty(B, dtype=torch.int32, device=dev)
@@ -295,7 +316,7 @@ def fef_loop_verification_inputs(tokens, window_pos, row_len, draft_tokens, stre
         _i32_cuda(t, "fef_loop_verification_inputs")
     B, L = tokens.shape
     K = window_pos.shape[1]
-    with torch.cuda.device(tokens.device):
+    with _on(tokens.device, stream):
         out = torch.empty((B, K, L), dtype=torch.int32, device=tokens.device)
         st = load().fef_loop_verification_inputs(tokens.data_ptr(), window_pos.data_ptr(), row_len.data_ptr(),
                                                  draft_tokens.data_ptr(), B, L, K, out.data_ptr(), _stream_ptr(stream))
@@ -310,7 +331,7 @@ def fef_loop_commit(window_pos, row_len, verified: "VerifyResult", tokens, conf,
         _i32_cuda(t, "fef_loop_commit")
     B, L = tokens.shape
     K = window_pos.shape[1]
-    with torch.cuda.device(tokens.device):
+    with _on(tokens.device, stream):
         committed = torch.empty(B, dtype=torch.int32, device=tokens.device)
         st = load().fef_loop_commit(window_pos.data_ptr(), row_len.data_ptr(), verified.accept_len.data_ptr(),
                                     verified.tokens.data_ptr(), verified.conf.data_ptr(), B, L, K, tokens.data_ptr(),
@@ -326,7 +347,7 @@ def fef_loop_advance_round(device_round: torch.Tensor, unresolved: Optional[torc
     _i32_cuda(device_round, "fef_loop_advance_round")
     if unresolved is not None:
         _i32_cuda(unresolved, "fef_loop_advance_round")
-    with torch.cuda.device(device_round.device):
+    with _on(device_round.device, stream):
         st = load().fef_loop_advance_round(device_round.data_ptr(),
                                            None if unresolved is None else unresolved.data_ptr(),
                                            0 if unresolved is None else unresolved.numel(), _stream_ptr(stream))
@@ -338,7 +359,7 @@ def fef_loop_remask(positions, count, tokens, conf, in_step, stream=None) -> Non
     """Send the selected positions back to MASK and empty the step's set (in place)."""
     B, L = tokens.shape
     k = positions.shape[1]
-    with torch.cuda.device(tokens.device):
+    with _on(tokens.device, stream):
         st = load().fef_loop_remask(positions.data_ptr() if k else None, count.data_ptr(), B, L, k, tokens.data_ptr(),
                                     conf.data_ptr(), in_step.data_ptr(), _stream_ptr(stream))
     if st != FEF_OK:
@@ -361,7 +382,7 @@ def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions:
         raise FefError(FEF_ERR_INVALID_ARG, "fef_remask_select")
     B, L = conf.shape
     dev = conf.device
-    with torch.cuda.device(dev):
+    with _on(dev, stream):
         if positions is None:
             positions = torch.empty((B, max(int(k), 0)), dtype=torch.int32, device=dev)
         if count is None:
@@ -393,7 +414,7 @@ def fef_spec_verify_static(draft_logits: torch.Tensor, target_logits: torch.Tens
     V = ld if V is None else int(V)
     code = _dtype_code(draft_logits)
     dev = draft_logits.device
-    with torch.cuda.device(dev):
+    with _on(dev, stream):
         if out is None:
             out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
                                torch.empty((B, K), dtype=torch.int32, device=dev),
@@ -441,7 +462,7 @@ def fef_spec_verify_host(draft_logits: torch.Tensor, target_logits: torch.Tensor
                                torch.empty((B, K), dtype=torch.int32).pin_memory(),
                                torch.empty((B, K), dtype=torch.float32).pin_memory(), 0)
     status = ctypes.c_int32(0)
-    with torch.cuda.device(arena.device):
+    with _on(arena.device, stream):
         st = load().fef_spec_verify_host(
             draft_logits.data_ptr(), target_logits.data_ptr(), draft_tokens.data_ptr(),
             None if row_len is None else row_len.data_ptr(), B, K, V, ld, code, float(temperature),
@@ -471,7 +492,7 @@ def fef_remask_select_host(conf: torch.Tensor, mask: torch.Tensor, k: int, arena
         positions = torch.empty((B, max(int(k), 0)), dtype=torch.int32).pin_memory()
     if count is None:
         count = torch.empty(B, dtype=torch.int32).pin_memory()
-    with torch.cuda.device(arena.device):
+    with _on(arena.device, stream):
         st = load().fef_remask_select_host(conf.data_ptr(), mask.data_ptr(), B, L, int(k),
                                            positions.data_ptr() if positions.numel() else None, count.data_ptr(),
                                            arena.data_ptr(), arena.numel(), _stream_ptr(stream))
@@ -484,3 +505,76 @@ __all__ = ["fef_loop_advance_round", "fef_loop_next_window", "fef_loop_verificat
            "fef_draft_sample", "fef_draft_sample_workspace_bytes", "DraftResult", "fef_spec_verify_static", "HostVerifyResult", "fef_spec_verify_host_arena_bytes", "fef_spec_verify_host",
            "fef_remask_select_host_arena_bytes", "fef_remask_select_host","load", "FefError", "VerifyResult", "fef_status_string", "fef_spec_verify_workspace_bytes",
            "fef_spec_verify", "fef_remask_select", "EXPORTS"]
+
+
+# ------------------------------------------------------------ verification from hidden states ----
+def fef_lmhead_verify_workspace_bytes(B: int, K: int, V: int, d: int) -> int:
+    return int(load().fef_lmhead_verify_workspace_bytes(B, K, V, d))
+
+
+def _bf16_matrix(t: torch.Tensor, where: str):
+    if t.device.type != "cuda" or t.dtype != torch.bfloat16 or t.dim() != 2 or not t.is_contiguous():
+        raise FefError(FEF_ERR_INVALID_ARG, where)
+    return t
+
+
+def fef_lmhead_verify(draft_hidden: torch.Tensor, target_hidden: torch.Tensor, weight: torch.Tensor,
+                      draft_tokens: torch.Tensor, temperature: float, seed: int, step: int,
+                      row_len: Optional[torch.Tensor] = None, out: Optional[VerifyResult] = None,
+                      workspace: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+    """Enqueue one verification call on hidden states (see ``fef_lmhead_verify`` in include/fef.h).
+
+    ``draft_hidden`` / ``target_hidden``: ``[B*K, d]`` bfloat16 CUDA tensors; ``weight``: ``[V, d]``
+    bfloat16; ``draft_tokens``: ``[B, K]`` int32.
+    """
+    for t in (draft_hidden, target_hidden, weight):
+        _bf16_matrix(t, "fef_lmhead_verify")
+    _require_cuda(draft_tokens, row_len)
+    if draft_tokens.dtype != torch.int32 or draft_tokens.dim() != 2 or not draft_tokens.is_contiguous():
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_lmhead_verify")
+    B, K = draft_tokens.shape
+    V, d = weight.shape
+    if draft_hidden.shape != (B * K, d) or target_hidden.shape != (B * K, d):
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_lmhead_verify")
+    if row_len is not None and row_len.dtype != torch.int32:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_lmhead_verify")
+    dev = weight.device
+    with _on(dev, stream):
+        if out is None:
+            out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.int32, device=dev),
+                               torch.empty((B, K), dtype=torch.float32, device=dev),
+                               torch.empty(1, dtype=torch.int32, device=dev))
+        if workspace is None:
+            workspace = torch.empty(max(fef_lmhead_verify_workspace_bytes(B, K, V, d), 256), dtype=torch.uint8, device=dev)
+        st = load().fef_lmhead_verify(draft_hidden.data_ptr(), target_hidden.data_ptr(), weight.data_ptr(),
+                                      draft_tokens.data_ptr(), None if row_len is None else row_len.data_ptr(),
+                                      B, K, V, d, float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                      int(step) & 0xFFFFFFFF, out.accept_len.data_ptr(), out.tokens.data_ptr(),
+                                      out.conf.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                      out.device_status.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_lmhead_verify")
+    return out
+
+
+def fef_lmhead_logits(hidden: torch.Tensor, weight: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):
+    """The binary32 logits ``hidden @ weight.T`` as the verification from hidden states sees them
+    (see ``fef_lmhead_logits`` in include/fef.h).  Returns ``(logits [rows, ldo] float32, device_status)``;
+    the first ``V`` entries of a row are the logits."""
+    _bf16_matrix(hidden, "fef_lmhead_logits")
+    _bf16_matrix(weight, "fef_lmhead_logits")
+    rows, d = hidden.shape
+    V = weight.shape[0]
+    if weight.shape[1] != d:
+        raise FefError(FEF_ERR_INVALID_ARG, "fef_lmhead_logits")
+    dev = weight.device
+    with _on(dev, stream):
+        if out is None:
+            out = torch.empty((rows, (V + 3) // 4 * 4), dtype=torch.float32, device=dev)
+        status = torch.empty(1, dtype=torch.int32, device=dev)
+        st = load().fef_lmhead_logits(hidden.data_ptr(), weight.data_ptr(), rows, V, d, out.data_ptr(), out.shape[1],
+                                      status.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_lmhead_logits")
+    return out, status

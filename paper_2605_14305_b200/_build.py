@@ -10,8 +10,9 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libfef.so")
-SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu", "fef_loop.cu"]
-HEADERS = [os.path.join(CSRC, "fef_common.cuh"), os.path.join(CSRC, "fef_device_math.cuh"), os.path.join(INCLUDE, "fef.h")]
+SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu", "fef_loop.cu", "fef_lmhead.cu"]
+HEADERS = [os.path.join(CSRC, h) for h in ("fef_common.cuh", "fef_device_math.cuh", "fef_verify_params.cuh",
+                                            "fef_residual.cuh")] + [os.path.join(INCLUDE, "fef.h")]
 
 
 def nvcc_path() -> str:
@@ -44,6 +45,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
+
+
+TEST_HOOKS_LIB_PATH = os.path.join(HERE, "libfef_testhooks.so")
+
+
+def build_test_hooks(force: bool = False) -> str:
+    """The library compiled with -DFEF_TEST_HOOKS (adds fef_test_withhold_stage_once, which lets a test
+    make one bounded wait of the streaming kernel run out).  Used by the GPU tests only."""
+    deps = [os.path.join(CSRC, s) for s in SOURCES] + HEADERS
+    if not force and os.path.exists(TEST_HOOKS_LIB_PATH) and \
+            all(os.path.getmtime(d) <= os.path.getmtime(TEST_HOOKS_LIB_PATH) for d in deps):
+        return TEST_HOOKS_LIB_PATH
+    tmp = TEST_HOOKS_LIB_PATH + ".tmp%d" % os.getpid()
+    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-DFEF_TEST_HOOKS",
+           "-I", INCLUDE, "-I", CSRC, "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+    subprocess.check_call(cmd)
+    os.replace(tmp, TEST_HOOKS_LIB_PATH)
+    return TEST_HOOKS_LIB_PATH
 
 
 if __name__ == "__main__":

@@ -17,7 +17,8 @@ constexpr int kChunkBytes = kConsumerWarps * 32 * 16 * kVecPerThread;  // 32 KiB
 constexpr int kHalves = 2;                              // chunks per tile: one barrier wait and one release per 64 KiB
 constexpr int kTileBytes = kChunkBytes * kHalves;       // 64 KiB
 constexpr int kStages = 3;                              // ring depth: 192 KiB in flight per SM
-constexpr int kSpinLimit = 1 << 22;                     // bound on every mbarrier wait loop
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;  // a wait inside a kernel gives up after this long (1 s)
+constexpr int kSpinRounds = 1 << 24;                    // ... or after this many rounds of 64 polls, whichever comes first
 constexpr int kSlotSets = 8;                            // in-CTA combine buffers (a warp leads by < 8 flushes)
 
 constexpr float kNoReference = -3.0e38f;                // "no reference yet" for the running softmax
@@ -45,9 +46,10 @@ struct __align__(16) ResidualTask {
     double kq;          // same for the draft law
 };
 
-// Counter shared by all CTAs of the streaming kernel (cleared by begin_call_kernel, the call's first kernel).
+// Shared by all CTAs of the streaming kernel (cleared by begin_call_kernel, the call's first kernel).
 struct __align__(16) Control {
     unsigned long long next_claim;  // next streaming claim to hand out
+    int aborted;                    // a bounded wait ran out: the partials are incomplete, no window is decided
 };
 
 // Vocabulary-parallel verification: what one rank reports for a rejected window after its
@@ -241,11 +243,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the limit ran out or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (int spin = 0; spin < kSpinLimit; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63) == 63 && *abort_flag) return false;
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when `limit_ns` of wall time have passed (the poll count is a second bound,
+// should the timer not advance) or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  unsigned long long limit_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long start = globaltimer_ns();
+    for (int round = 0; round < kSpinRounds; ++round) {
+        for (int spin = 0; spin < 64; ++spin)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - start > limit_ns) return false;
     }
     return false;
 }

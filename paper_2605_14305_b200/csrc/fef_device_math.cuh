@@ -149,6 +149,17 @@ struct Top2 {
     }
 };
 
+__device__ __forceinline__ double warp_max(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
 // The three largest (weight, lowest id) a thread, warp or CTA has seen; empty slots hold weight 0.
 struct Top3 {
     float w1, w2, w3;
@@ -175,18 +186,34 @@ struct Top3 {
             x3 = x;
         }
     }
-    // best three of the whole warp, in every lane
+    // Best three of the whole warp, in every lane: three rounds of "largest head over the lanes wins and
+    // its lane moves on to its next entry" (weights are >= 0, so their bit patterns order like the values;
+    // among equal weights the lowest id wins, as in offer()).
     __device__ __forceinline__ void warp_merge() {
+        float rw[3];
+        int rx[3];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ow1 = __shfl_xor_sync(0xFFFFFFFFu, w1, o), ow2 = __shfl_xor_sync(0xFFFFFFFFu, w2, o);
-            const float ow3 = __shfl_xor_sync(0xFFFFFFFFu, w3, o);
-            const int ox1 = __shfl_xor_sync(0xFFFFFFFFu, x1, o), ox2 = __shfl_xor_sync(0xFFFFFFFFu, x2, o);
-            const int ox3 = __shfl_xor_sync(0xFFFFFFFFu, x3, o);
-            offer(ow1, ox1);
-            offer(ow2, ox2);
-            offer(ow3, ox3);
+        for (int r = 0; r < 3; ++r) {
+            const unsigned head = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(w1));
+            const bool holder = __float_as_uint(w1) == head;
+            const int id = __reduce_min_sync(0xFFFFFFFFu, holder ? x1 : 0x7FFFFFFF);
+            rw[r] = __uint_as_float(head);
+            rx[r] = id;
+            if (holder && x1 == id) {
+                w1 = w2;
+                x1 = x2;
+                w2 = w3;
+                x2 = x3;
+                w3 = 0.f;
+                x3 = 0x7FFFFFFF;
+            }
         }
+        w1 = rw[0];
+        x1 = rx[0];
+        w2 = rw[1];
+        x2 = rx[1];
+        w3 = rw[2];
+        x3 = rx[2];
     }
 };
 

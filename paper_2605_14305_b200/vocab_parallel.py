@@ -11,8 +11,7 @@ from typing import List, Optional, Sequence, Tuple
 
 import torch
 
-from . import (FEF_ERR_INVALID_ARG, FEF_OK, FefError, VerifyResult, _dtype_code, _require_cuda, _stream_ptr,
-               fef_spec_verify_workspace_bytes, load)
+from . import FEF_ERR_INVALID_ARG, FEF_OK, FefError, VerifyResult, _dtype_code, _require_cuda, _stream_ptr, load
 
 STATS_PER_ROW = 6
 CANDIDATE_BYTES = 16
@@ -38,8 +37,10 @@ def shard_vocab(V: int, ranks: int, multiple: int = 8) -> List[Tuple[int, int]]:
 class _Rank:
     """Buffers and sizes of one rank's slice."""
 
-    def __init__(self, q: torch.Tensor, p: torch.Tensor, offset: int, V_local: Optional[int]):
-        _require_cuda(q, p)
+    def __init__(self, q: torch.Tensor, p: torch.Tensor, offset: int, V_local: Optional[int], lib=None):
+        self.lib = load() if lib is None else lib   # (a stand-in library object is only given by host-side tests)
+        if lib is None:
+            _require_cuda(q, p)
         if q.dim() != 3 or q.shape != p.shape or q.dtype != p.dtype or not (q.is_contiguous() and p.is_contiguous()):
             raise FefError(FEF_ERR_INVALID_ARG, "fef_vp_local_stats")
         self.q, self.p, self.offset = q, p, int(offset)
@@ -47,12 +48,17 @@ class _Rank:
         self.V = self.ld if V_local is None else int(V_local)
         self.code = _dtype_code(q)
         dev = q.device
-        self.workspace = torch.empty(max(fef_spec_verify_workspace_bytes(self.B, self.K, self.V, self.code), 256),
-                                     dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(max(int(self.lib.fef_spec_verify_workspace_bytes(self.B, self.K, self.V, self.code)),
+                                         256), dtype=torch.uint8, device=dev)
         self.stats = torch.empty((self.B * self.K, STATS_PER_ROW), dtype=torch.float64, device=dev)
-        self.tasks = torch.empty(int(load().fef_vp_task_bytes(self.B)), dtype=torch.uint8, device=dev)
+        self.tasks = torch.empty(int(self.lib.fef_vp_task_bytes(self.B)), dtype=torch.uint8, device=dev)
         self.cand = torch.zeros((self.B, CANDIDATE_BYTES), dtype=torch.uint8, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+
+def _sptr(stream) -> int:
+    # (a host-side test with a stand-in library and no CUDA device has no stream to name)
+    return 0 if stream is None and not torch.cuda.is_available() else _stream_ptr(stream)
 
 
 def _check(st: int, where: str):
@@ -61,30 +67,30 @@ def _check(st: int, where: str):
 
 
 def _local_stats(r: _Rank, tokens, row_len, T, stream):
-    _check(load().fef_vp_local_stats(r.q.data_ptr(), r.p.data_ptr(), tokens.data_ptr(),
+    _check(r.lib.fef_vp_local_stats(r.q.data_ptr(), r.p.data_ptr(), tokens.data_ptr(),
                                      None if row_len is None else row_len.data_ptr(), r.B, r.K, r.V, r.ld, r.code,
                                      float(T), r.offset, r.stats.data_ptr(), r.workspace.data_ptr(),
-                                     r.workspace.numel(), r.status.data_ptr(), _stream_ptr(stream)), "fef_vp_local_stats")
+                                     r.workspace.numel(), r.status.data_ptr(), _sptr(stream)), "fef_vp_local_stats")
 
 
 def _accept(r: _Rank, stats_all, ranks, tokens, row_len, V_total, T, seed, step, out: VerifyResult, stream):
-    _check(load().fef_vp_accept(stats_all.data_ptr(), ranks, tokens.data_ptr(),
+    _check(r.lib.fef_vp_accept(stats_all.data_ptr(), ranks, tokens.data_ptr(),
                                 None if row_len is None else row_len.data_ptr(), r.B, r.K, int(V_total), r.code, float(T),
                                 int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF, out.accept_len.data_ptr(),
                                 out.tokens.data_ptr(), out.conf.data_ptr(), r.tasks.data_ptr(),
-                                out.device_status.data_ptr(), _stream_ptr(stream)), "fef_vp_accept")
+                                out.device_status.data_ptr(), _sptr(stream)), "fef_vp_accept")
 
 
 def _local_residual(r: _Rank, T, seed, step, stream):
-    _check(load().fef_vp_local_residual(r.q.data_ptr(), r.p.data_ptr(), r.tasks.data_ptr(), r.B, r.K, r.V, r.ld, r.code,
+    _check(r.lib.fef_vp_local_residual(r.q.data_ptr(), r.p.data_ptr(), r.tasks.data_ptr(), r.B, r.K, r.V, r.ld, r.code,
                                         float(T), int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF, r.offset,
                                         r.cand.data_ptr(), r.workspace.data_ptr(), r.workspace.numel(),
-                                        _stream_ptr(stream)), "fef_vp_local_residual")
+                                        _sptr(stream)), "fef_vp_local_residual")
 
 
 def _finish(r: _Rank, cand_all, ranks, T, out: VerifyResult, stream):
-    _check(load().fef_vp_finish(cand_all.data_ptr(), ranks, r.tasks.data_ptr(), r.B, r.K, r.code, float(T),
-                                out.tokens.data_ptr(), out.conf.data_ptr(), _stream_ptr(stream)), "fef_vp_finish")
+    _check(r.lib.fef_vp_finish(cand_all.data_ptr(), ranks, r.tasks.data_ptr(), r.B, r.K, r.code, float(T),
+                                out.tokens.data_ptr(), out.conf.data_ptr(), _sptr(stream)), "fef_vp_finish")
 
 
 def _new_result(B, K, dev) -> VerifyResult:
@@ -95,26 +101,34 @@ def _new_result(B, K, dev) -> VerifyResult:
 def fef_spec_verify_vocab_parallel(draft_slice: torch.Tensor, target_slice: torch.Tensor, draft_tokens: torch.Tensor,
                                    temperature: float, seed: int, step: int, vocab_offset: int, V_total: int,
                                    row_len: Optional[torch.Tensor] = None, V_local: Optional[int] = None,
-                                   group=None, stream=None) -> VerifyResult:
+                                   group=None, stream=None, lib=None) -> VerifyResult:
     """One verification call on this rank of a ``torch.distributed`` group whose ranks hold the
     slices of the vocabulary (``draft_slice`` / ``target_slice``: ``[B, K, ld_local]``).  Every
     rank returns the same result.  ``device_status`` holds the acceptance step's status; a
-    streaming-side error of this rank is raised into it as well."""
+    streaming-side error of this rank is raised into it as well.
+
+    The kernels, the two all-gathers and every allocation of the call run on ``stream`` (made the
+    current stream for the duration of the call), so they are ordered against each other whichever
+    stream the caller was on.  ``lib``: a stand-in for the loaded library (host-side tests only)."""
+    import contextlib
+
     import torch.distributed as dist
 
     ranks = dist.get_world_size(group)
-    r = _Rank(draft_slice, target_slice, vocab_offset, V_local)
-    out = _new_result(r.B, r.K, draft_slice.device)
-    _local_stats(r, draft_tokens, row_len, temperature, stream)
-    # (gathered by concatenation along the first axis: rank-major, the layout the next call reads)
-    stats_all = torch.empty((ranks * r.stats.shape[0], STATS_PER_ROW), dtype=torch.float64, device=r.stats.device)
-    dist.all_gather_into_tensor(stats_all, r.stats, group=group)
-    _accept(r, stats_all, ranks, draft_tokens, row_len, V_total, temperature, seed, step, out, stream)
-    _local_residual(r, temperature, seed, step, stream)
-    cand_all = torch.empty((ranks * r.B, CANDIDATE_BYTES), dtype=torch.uint8, device=r.cand.device)
-    dist.all_gather_into_tensor(cand_all, r.cand, group=group)
-    _finish(r, cand_all, ranks, temperature, out, stream)
-    torch.maximum(out.device_status, r.status, out=out.device_status)
+    on_stream = torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
+    with on_stream:
+        r = _Rank(draft_slice, target_slice, vocab_offset, V_local, lib)
+        out = _new_result(r.B, r.K, draft_slice.device)
+        _local_stats(r, draft_tokens, row_len, temperature, stream)
+        # (gathered by concatenation along the first axis: rank-major, the layout the next call reads)
+        stats_all = torch.empty((ranks * r.stats.shape[0], STATS_PER_ROW), dtype=torch.float64, device=r.stats.device)
+        dist.all_gather_into_tensor(stats_all, r.stats, group=group)
+        _accept(r, stats_all, ranks, draft_tokens, row_len, V_total, temperature, seed, step, out, stream)
+        _local_residual(r, temperature, seed, step, stream)
+        cand_all = torch.empty((ranks * r.B, CANDIDATE_BYTES), dtype=torch.uint8, device=r.cand.device)
+        dist.all_gather_into_tensor(cand_all, r.cand, group=group)
+        _finish(r, cand_all, ranks, temperature, out, stream)
+        torch.maximum(out.device_status, r.status, out=out.device_status)
     return out
 
 

@@ -252,3 +252,105 @@ def test_decode_loop_driver_with_the_oracle_as_backend():
     # after the first denoising step only the k re-masked positions per row are unresolved
     first_redo = next(i for i, c in enumerate(calls) if i > 0 and (c == k).all() and (calls[i - 1] != k).any())
     assert first_redo >= L // w.K
+
+
+_VP_WORKER = r"""
+import ctypes, json, sys
+sys.path.insert(0, %r)
+import torch, torch.distributed as dist
+from paper_2605_14305_b200 import vocab_parallel as vp
+
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+B, K, Vloc = 3, 4, 16
+
+
+class FakeLibrary:
+    # Stand-in for the loaded library: records the order of the calls, fills this rank's outputs with
+    # values that name the rank, and checks what the gathers hand to the next step.
+    def __init__(self):
+        self.calls = []
+
+    def fef_spec_verify_workspace_bytes(self, B_, K_, V_, code):
+        return 4096
+
+    def fef_vp_task_bytes(self, B_):
+        return 32 * B_
+
+    def _view(self, ptr, n, ctype):
+        return (ctype * n).from_address(ptr)
+
+    def fef_vp_local_stats(self, q, p, tok, row_len, B_, K_, V_, ld, code, T, offset, stats, ws, wsb, status, stream):
+        self.calls.append("stats")
+        assert (B_, K_, V_, ld) == (B, K, Vloc, Vloc) and offset == rank * Vloc and wsb >= 4096 and stream == 0
+        s = self._view(stats, B * K * vp.STATS_PER_ROW, ctypes.c_double)
+        for i in range(len(s)):
+            s[i] = 1000.0 * rank + i
+        return 0
+
+    def fef_vp_accept(self, stats_all, ranks, tok, row_len, B_, K_, V_total, code, T, seed, step, accept_len, tokens, conf,
+                      tasks, status, stream):
+        self.calls.append("accept")
+        assert ranks == world and V_total == world * Vloc and (seed, step) == (77, 5)
+        n = B * K * vp.STATS_PER_ROW
+        s = self._view(stats_all, world * n, ctypes.c_double)
+        for r in range(world):          # rank-major: rank r's block follows rank r - 1's
+            assert s[r * n] == 1000.0 * r and s[r * n + n - 1] == 1000.0 * r + n - 1
+        a = self._view(accept_len, B, ctypes.c_int32)
+        for b in range(B):
+            a[b] = b
+        return 0
+
+    def fef_vp_local_residual(self, q, p, tasks, B_, K_, V_, ld, code, T, seed, step, offset, cand, ws, wsb, stream):
+        self.calls.append("residual")
+        assert offset == rank * Vloc and (seed, step) == (77, 5)
+        c = self._view(cand, B * vp.CANDIDATE_BYTES, ctypes.c_uint8)
+        for i in range(len(c)):
+            c[i] = (17 * rank + i) %% 251
+        return 0
+
+    def fef_vp_finish(self, cand_all, ranks, tasks, B_, K_, code, T, tokens, conf, stream):
+        self.calls.append("finish")
+        assert ranks == world
+        n = B * vp.CANDIDATE_BYTES
+        c = self._view(cand_all, world * n, ctypes.c_uint8)
+        for r in range(world):
+            assert c[r * n] == (17 * r) %% 251 and c[r * n + n - 1] == (17 * r + n - 1) %% 251
+        return 0
+
+
+lib = FakeLibrary()
+q = torch.zeros((B, K, Vloc))
+tok = torch.zeros((B, K), dtype=torch.int32)
+out = vp.fef_spec_verify_vocab_parallel(q, q.clone(), tok, 1.0, 77, 5, rank * Vloc, world * Vloc, lib=lib)
+assert lib.calls == ["stats", "accept", "residual", "finish"], lib.calls
+assert out.accept_len.tolist() == [0, 1, 2]
+if rank == 0:
+    print(json.dumps({"ok": True}))
+"""
+
+
+def test_vocab_parallel_orchestration_over_gloo_with_a_stand_in_library(tmp_path):
+    """The four steps of the vocabulary-parallel call and its two all-gathers, driven on two CPU
+    ranks (gloo) with a stand-in for the library: call order, arguments, and the rank-major layout
+    of what each gather hands to the following step."""
+    script = tmp_path / "vp_worker.py"
+    script.write_text(_VP_WORKER % ROOT)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(script)]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=240, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-3000:]
+    assert json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])["ok"]
+
+
+def test_bench_gpus_flag_starts_ranks_itself(tmp_path):
+    """`bench.py --gpus 2` run by hand (no WORLD_SIZE) re-launches itself as two ranks; rank 0 alone prints."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny", "--steps", "2",
+           "--warmup", "1", "--gpus", "2"]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=240, cwd=ROOT, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and "parallelism" in d and "parallelism" not in d["config"]

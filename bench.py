@@ -249,7 +249,7 @@ def run_native(args):
                 stage_ms[j] += evs[j].elapsed_time(evs[j + 1])
         stage_ms = [x / steps for x in stage_ms]
     # timed region 4 (not part of the step): the draft-token draws that precede a verification call
-    draft_ms = norm_ms = None
+    draft_ms = norm_ms = both_ms = round_ms = None
     if not args.no_call_events:
         dws = torch.empty(max(fef.fef_draft_sample_workspace_bytes(w.B, w.K, w.V, w.dtype), 256), dtype=torch.uint8,
                           device=dev)
@@ -273,6 +273,25 @@ def run_native(args):
         d1.record(stream)
         barrier()
         norm_ms = d0.elapsed_time(d1) / steps
+        # ... and a whole round with both tensors read once: draft draws that also reduce the target rows, then
+        # the verification that takes both normalisers (it streams nothing)
+        dboth = fef.fef_draft_sample(sets[0][0], w.temperature, seed, 0, workspace=dws, target_logits=sets[0][1])
+        barrier()
+        d0.record(stream)
+        for i in range(steps):
+            q, p, _ = sets[i % nbuf]
+            fef.fef_draft_sample(q, w.temperature, seed, i, out=dboth, workspace=dws, target_logits=p)
+        d1.record(stream)
+        for i in range(steps):
+            q, p, _ = sets[i % nbuf]
+            fef.fef_draft_sample(q, w.temperature, seed, i, out=dboth, workspace=dws, target_logits=p)
+            fef.fef_spec_verify(q, p, dboth.tokens, w.temperature, seed, i, out=out, workspace=ws,
+                                draft_log2_norm=dboth.log2_norm, target_log2_norm=dboth.target_log2_norm)
+        d2 = torch.cuda.Event(enable_timing=True)
+        d2.record(stream)
+        barrier()
+        both_ms = d0.elapsed_time(d1) / steps
+        round_ms = d1.elapsed_time(d2) / steps
     sampler.stop()
     status = int(out.device_status.item())
     accept_mean = float(out.accept_len.float().mean().item())
@@ -384,7 +403,13 @@ def run_native(args):
             "note": "fef_draft_sample on the draft logits of the same workload; bound by Philox arithmetic, not "
                     "by HBM; not part of the step",
             "verify_with_draft_norm_ms": norm_ms,
-            "verify_with_draft_norm_positions_per_s": w.B * w.K / (norm_ms * 1e-3)},
+            "verify_with_draft_norm_positions_per_s": w.B * w.K / (norm_ms * 1e-3),
+            "draft_sample_with_target_ms": both_ms,
+            "round_ms": round_ms,
+            "round_note": "fef_draft_sample with the target logits + fef_spec_verify with both normalisers: one "
+                          "whole round of Algorithm 2 (draws, verification), both tensors read once",
+            "round_positions_per_s": w.B * w.K / (round_ms * 1e-3),
+            "round_gbs": 2 * w.B * w.K * w.V * w.logit_bytes / (round_ms * 1e-3) / 1e9},
         # per step: begin-call, streaming, tail (acceptance tests + residual draw; greedy: scan), re-mask kernels
         "gpu_launches": steps * 4,
         "clocks": sampler.result(),
@@ -438,39 +463,140 @@ def run_reference(args):
 
 # ------------------------------------------------------------- loop sweep ----
 def run_loop_sweep(args):
-    """Extra mode (not the contract's line): the long-generation sweep — the full decoding loop
-    (window, draft draws, verification, commit; re-masking between two denoising steps) on a
-    device-resident state of L = 1024 positions per sequence until nothing is masked, at
-    B in {1, 8, 64} x K in {8, 32, 64}, bf16 and fp32, eager and as a replayed CUDA graph.
-    The logits are fixed tensors made before the loop (their generation is not in the time)."""
+    """Extra mode (not the contract's line): the long-generation sweep.  The full decoding loop
+    (window, logits, draft draws that also reduce the target rows, verification with both
+    normalisers, commit; LowConf and re-masking between the denoising steps) on a device-resident
+    state of L = 1024 positions per sequence until nothing is masked, at B in {1, 8, 64} x
+    K in {8, 32, 64}, bf16 and fp32.  The logits of every round are made on the device from a seeded
+    Philox stream (target = draft + N(0, 0.7^2)) inside the round; the generator's own time per
+    round is measured separately and reported beside the round time.  "eager": the host drives the
+    rounds and reads one integer per round; "graph": the whole loop is one graph launch
+    (fef_loop_run_synthetic: a WHILE node around the round, no host in between)."""
     import paper_2605_14305_b200 as fef
-    from paper_2605_14305_b200.decode_loop import run_decode_loop_device, run_decode_loop_graph
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device
 
     fef.load(build_if_missing=True)
     torch.cuda.set_device(0)
-    L, remask_k = 1024, 8
+    L, remask_k, steps, V, T = 1024, 8, 2, synth.HEADLINE.V, 1.0
     points = []
     for dtype in (torch.bfloat16, torch.float32):
         for B in (1, 8, 64):
             for K in (8, 32, 64):
-                w = synth.HEADLINE.with_(B=B, K=K, dtype=dtype, noise_std=0.7)
-                t0 = time.perf_counter()
-                q, p = synth.make_logits(w, seed=args.seed, device="cuda")
+                def logits_fn(rnd, window, row_len, inputs):
+                    return fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, args.seed, rnd, boost_fraction=0.01, boost=8.0)
+
+                # the generator alone
+                buf = logits_fn(0, None, None, None)
                 torch.cuda.synchronize()
-                gen_s = time.perf_counter() - t0
-                res = {}
-                for name, fn, lf in (("eager", run_decode_loop_device, lambda rnd, window, row_len, inputs: (q, p)),
-                                     ("graph", run_decode_loop_graph, lambda rnd, window, row_len: (q, p))):
-                    fn(fef, B, L, K, 2, remask_k, lf, w.temperature, args.seed)       # warm-up
-                    out = fn(fef, B, L, K, 2, remask_k, lf, w.temperature, args.seed)
-                    res[name] = {"rounds": out["rounds"], "us_per_round": out["loop_seconds"] * 1e6 / out["rounds"],
-                                 "committed_positions_per_s": (B * L + B * remask_k) / out["loop_seconds"]}
-                points.append({"B": B, "K": K, "dtype": "bf16" if dtype == torch.bfloat16 else "f32",
-                               "logit_generation_s": gen_s, **res})
-                del q, p
-    print(json.dumps({"mode": "loop sweep", "L": L, "V": synth.HEADLINE.V, "denoising_steps": 2, "remask_k": remask_k,
-                      "verification": "fef_draft_sample + fef_spec_verify reusing the draft normalisers",
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record()
+                for r in range(10):
+                    fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, args.seed, r, boost_fraction=0.01, boost=8.0, out=buf)
+                g1.record()
+                torch.cuda.synchronize()
+                gen_us = g0.elapsed_time(g1) * 1e3 / 10
+                del buf
+                run_decode_loop_device(fef, B, L, K, steps, remask_k, logits_fn, T, args.seed, reuse_target_norm=True, V=V)
+                eager = run_decode_loop_device(fef, B, L, K, steps, remask_k, logits_fn, T, args.seed,
+                                               reuse_target_norm=True, V=V)
+                fef.fef_loop_run_synthetic(B, L, K, V, dtype, T, args.seed, steps, remask_k, 2.0, 0.7, 0.01, 8.0)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                graph = fef.fef_loop_run_synthetic(B, L, K, V, dtype, T, args.seed, steps, remask_k, 2.0, 0.7, 0.01, 8.0)
+                torch.cuda.synchronize()
+                graph_s = time.perf_counter() - t0
+                same = bool((graph["tokens"] == eager["tokens"]).all().item()) and graph["rounds"] == eager["rounds"]
+                rounds = eager["rounds"]
+                points.append({
+                    "B": B, "K": K, "dtype": "bf16" if dtype == torch.bfloat16 else "f32", "rounds": rounds,
+                    "generator_us_per_round": gen_us,
+                    "eager_us_per_round": eager["loop_seconds"] * 1e6 / rounds,
+                    "graph_us_per_round": graph_s * 1e6 / rounds,
+                    "graph_us_per_round_without_generator": graph_s * 1e6 / rounds - gen_us,
+                    "committed_positions_per_s_graph": (B * L + B * remask_k) / graph_s,
+                    "graph_equals_eager": same})
+    print(json.dumps({"mode": "loop sweep", "L": L, "V": V, "denoising_steps": steps, "remask_k": remask_k,
+                      "round": "fef_synth_logits + fef_draft_sample_with_target + fef_spec_verify_with_norms + bookkeeping",
+                      "note": "graph time includes building and instantiating the graph (once per loop)",
                       "data": "synthetic", "points": points}))
+
+
+# ------------------------------------------------------- from hidden states ----
+def run_lmhead(args):
+    """Extra mode (not the contract's line): verification straight from hidden states
+    (``fef_lmhead_verify``: output-layer product on the tensor cores with the softmax partials in its
+    epilogue) at the headline window shape with a hidden width of ``--d`` (default 4096), against a
+    tensor-core roofline; beside it the unfused path: two library products that write bfloat16 logits,
+    then ``fef_spec_verify`` on them."""
+    import paper_2605_14305_b200 as fef
+
+    fef.load(build_if_missing=True)
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = _workload(args)
+    B, K, V, d, T = w.B, w.K, w.V, args.d, w.temperature if w.temperature > 0 else 1.0
+    g = torch.Generator(device=dev).manual_seed(args.seed)
+    Hq = torch.randn((B * K, d), generator=g, device=dev)
+    Hp = (Hq + 0.35 * torch.randn((B * K, d), generator=g, device=dev)).to(torch.bfloat16)
+    Hq = Hq.to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=g, device=dev) * (2.0 / math.sqrt(d))).to(torch.bfloat16)
+    lq = Hq @ W.T
+    tok = synth.sample_draft_tokens(lq.view(B, K, V), T, args.seed + 1)
+    ws = torch.empty(fef.fef_lmhead_verify_workspace_bytes(B, K, V, d), dtype=torch.uint8, device=dev)
+    out = fef.fef_lmhead_verify(Hq, Hp, W, tok, T, args.seed, 0, workspace=ws)
+    ws2 = torch.empty(fef.fef_spec_verify_workspace_bytes(B, K, V, torch.bfloat16), dtype=torch.uint8, device=dev)
+    lp = torch.empty_like(lq)
+    out2 = fef.fef_spec_verify(lq.view(B, K, V), lq.view(B, K, V), tok, T, args.seed, 0, workspace=ws2)
+    steps, warmup = min(args.steps, 50), max(3, min(args.warmup, 5))
+    sampler = ClockSampler(0)
+    sampler.start()
+
+    def timed(fn):
+        for i in range(warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for i in range(steps):
+            fn(warmup + i)
+        t1.record()
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / steps
+
+    fused_ms = timed(lambda i: fef.fef_lmhead_verify(Hq, Hp, W, tok, T, args.seed, i, out=out, workspace=ws))
+
+    def unfused(i):
+        torch.matmul(Hq, W.T, out=lq)
+        torch.matmul(Hp, W.T, out=lp)
+        fef.fef_spec_verify(lq.view(B, K, V), lp.view(B, K, V), tok, T, args.seed, i, out=out2, workspace=ws2)
+
+    unfused_ms = timed(unfused)
+    gemm_ms = timed(lambda i: (torch.matmul(Hq, W.T, out=lq), torch.matmul(Hp, W.T, out=lp)))
+    sampler.stop()
+    status = int(out.device_status.item())
+    same = bool((out.accept_len == out2.accept_len).float().mean().item() > 0.9)
+    flops_stats = 2.0 * 2 * B * K * d * V
+    flops_all = flops_stats + 2.0 * 2 * B * d * V
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, src = float(json.load(f)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json, sustained bf16 GEMM)"
+    except Exception:
+        peak, src = 1400.0, "fallback (earlier measurement on this pool, sustained)"
+    line = {
+        "mode": "verification from hidden states", "metric": METRIC, "unit": UNIT, "data": "synthetic", "dtype": "bf16",
+        "config": {"workload": "B=%d windows x K=%d positions, hidden width %d, V=%d, bf16 hidden states and weight, T=%g"
+                               % (B, K, d, V, T)},
+        "value": B * K / (fused_ms * 1e-3), "ms_per_step": fused_ms, "steps": steps, "warmup": warmup,
+        "roofline": {"bound": "tensor", "kernel": "lmhead_gemm_kernel", "unit": "TFLOP/s", "peak": peak, "peak_source": src,
+                     "achieved": flops_all / (fused_ms * 1e-3) / 1e12, "frac": flops_all / (fused_ms * 1e-3) / 1e12 / peak,
+                     "flops_per_call": flops_all, "traffic": None,
+                     "note": "whole call (both products, acceptance, the rejected rows' product, residual draw)"},
+        "unfused": {"ms_per_step": unfused_ms, "library_products_ms": gemm_ms,
+                    "library_tflops": flops_stats / (gemm_ms * 1e-3) / 1e12,
+                    "note": "torch.matmul to bfloat16 logits twice, then fef_spec_verify"},
+        "device_status": status, "accept_len_mostly_equal_to_unfused": same, "clocks": sampler.result(),
+    }
+    print(json.dumps(line))
 
 
 def main():
@@ -493,6 +619,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-call-events", action="store_true")
     ap.add_argument("--loop-sweep", action="store_true", help="time the full decoding loop at the sweep points instead")
+    ap.add_argument("--lmhead", action="store_true", help="time verification from hidden states (tensor-core product) instead")
+    ap.add_argument("--d", type=int, default=4096, help="hidden width for --lmhead")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.loop_sweep:
         # started by hand for several GPUs: become one rank per GPU (the same launch the driver uses)
@@ -500,7 +628,9 @@ def main():
         os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node",
                                    str(args.gpus), "--master-addr", "127.0.0.1", "--master-port", port,
                                    os.path.abspath(__file__)] + sys.argv[1:])
-    if args.loop_sweep:
+    if args.lmhead:
+        run_lmhead(args)
+    elif args.loop_sweep:
         run_loop_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

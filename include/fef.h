@@ -251,6 +251,35 @@ fef_status fef_draft_sample(const void* draft_logits, const int32_t* row_len,
                             int32_t* device_status, void* cuda_stream);
 
 /*
+ * Draft draws and the target laws' normalisers in one pass (Algorithm 2: the draft tokens are drawn
+ * from rho, then the target laws pi are needed at them): fef_draft_sample that reads the target
+ * logits of the same rows alongside and also returns
+ *   target_log2_norm  device out, [B, K] float64: log2 of sum_x 2^(l^p_x * log2(e) / T) per position
+ *                     (NaN where the target row holds NaN or +inf or no finite logit; 0 for i >= n_b),
+ * so that both tensors are read once, by one kernel.  fef_spec_verify_with_norms then verifies
+ * without streaming anything: it takes both normalisers, reads the two logits at each draft token and
+ * the rejected position's rows for the residual draw.  Results equal fef_spec_verify's up to the
+ * rounding of the normalisers (confidences within 1e-5 relative, the same draws apart from
+ * near-ties).  device_round: NULL, or the device-resident round counter of the *_at_round calls.
+ * At temperature 0 fef_spec_verify_with_norms ignores the normalisers and runs as fef_spec_verify does.
+ * Workspaces: fef_draft_sample_workspace_bytes / fef_spec_verify_workspace_bytes.
+ */
+fef_status fef_draft_sample_with_target(const void* draft_logits, const void* target_logits, const int32_t* row_len,
+                                        int B, int K, int V, int64_t ld, fef_dtype dt,
+                                        float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                        int32_t* draft_tokens, double* draft_log2_norm, double* target_log2_norm,
+                                        void* workspace, size_t workspace_bytes,
+                                        int32_t* device_status, void* cuda_stream);
+fef_status fef_spec_verify_with_norms(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                                      const double* draft_log2_norm, const double* target_log2_norm,
+                                      const int32_t* row_len,
+                                      int B, int K, int V, int64_t ld, fef_dtype dt,
+                                      float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                      int32_t* accept_len, int32_t* tokens, float* conf,
+                                      void* workspace, size_t workspace_bytes,
+                                      int32_t* device_status, void* cuda_stream);
+
+/*
  * LowConf_k of Algorithm 2 (the selection of the n_rm least confident positions of C^(s)
  * at the end of a denoising step): for every batch row the k candidate positions of lowest
  * confidence.
@@ -428,6 +457,42 @@ fef_status fef_lmhead_verify(const void* draft_hidden, const void* target_hidden
                              int32_t* device_status, void* cuda_stream);
 fef_status fef_lmhead_logits(const void* hidden, const void* weight, int rows, int V, int d,
                              float* logits, int64_t ldo, int32_t* device_status, void* cuda_stream);
+
+/*
+ * Seeded synthetic logits made on the device (benchmarks and tests of the decoding loop; they stand
+ * in for the two model calls of Algorithm 2 and hold none of the method's arithmetic):
+ *   draft  = draft_std * N(0,1), plus `boost` with probability boost_fraction (in steps of 1/512),
+ *   target = draft + noise_std * N(0,1),
+ * every element a pure function of (seed, round + *device_round, row, vocabulary id) through
+ * Philox4x32-10 and Box-Muller, rounded to the storage type.  [B, K, ld] row-major as in
+ * fef_spec_verify; ld must cover whole 16-byte vectors (ld >= V rounded up to 8 bfloat16 / 4 float32
+ * elements): the entries between V and that bound are written too.  device_round may be NULL.
+ */
+fef_status fef_synth_logits(void* draft_logits, void* target_logits, int B, int K, int V, int64_t ld, fef_dtype dt,
+                            float draft_std, float noise_std, float boost_fraction, float boost,
+                            uint64_t seed, uint32_t round, const uint32_t* device_round, void* cuda_stream);
+
+/*
+ * The whole decoding loop of Algorithm 2 as ONE submission, with fef_synth_logits in the place of
+ * the two model calls: n_steps denoising steps over B sequences of L positions; every round is
+ * window -> (at the end of a step: LowConf_k and re-masking) -> logits -> draft draws with the target
+ * normalisers -> verification -> commit, until nothing is unresolved after the last step.  The
+ * rounds are the body of a CUDA graph WHILE node whose condition a kernel of the round sets, so the
+ * host neither reads anything back nor submits anything between rounds.
+ *   tokens, conf, in_step  device, [B, L]: the state; pass all positions masked (FEF_MASK_TOKEN, -1, 0)
+ *                          to decode from scratch
+ *   device_round           device, [1] uint32: the round counter (random numbers of round r use step r);
+ *                          start it at 0; on return it holds the number of rounds run
+ *   L <= FEF_MAX_REMASK_L; temperature > 0; remask_k >= 0
+ *   workspace              fef_loop_run_synthetic_workspace_bytes(...) bytes (it holds the two logit
+ *                          tensors of a round), 256-byte aligned
+ * The call builds, launches and destroys the graph and returns after synchronising `cuda_stream`.
+ */
+size_t fef_loop_run_synthetic_workspace_bytes(int B, int L, int K, int V, fef_dtype dt, int remask_k);
+fef_status fef_loop_run_synthetic(int B, int L, int K, int V, fef_dtype dt, float temperature, uint64_t seed,
+                                  int n_steps, int remask_k, float draft_std, float noise_std, float boost_fraction,
+                                  float boost, int32_t* tokens, float* conf, uint8_t* in_step, uint32_t* device_round,
+                                  void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
 #ifdef __cplusplus
 }

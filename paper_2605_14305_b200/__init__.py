@@ -30,7 +30,9 @@ EXPORTS = ("fef_status_string", "fef_spec_verify_workspace_bytes", "fef_spec_ver
            "fef_loop_next_window", "fef_loop_verification_inputs", "fef_loop_commit", "fef_loop_remask",
            "fef_draft_sample_at_round", "fef_spec_verify_at_round", "fef_loop_advance_round",
            "fef_vp_task_bytes", "fef_vp_local_stats", "fef_vp_accept", "fef_vp_local_residual", "fef_vp_finish",
-           "fef_lmhead_verify_workspace_bytes", "fef_lmhead_verify", "fef_lmhead_logits")
+           "fef_lmhead_verify_workspace_bytes", "fef_lmhead_verify", "fef_lmhead_logits",
+           "fef_draft_sample_with_target", "fef_spec_verify_with_norms", "fef_synth_logits",
+           "fef_loop_run_synthetic_workspace_bytes", "fef_loop_run_synthetic")
 
 _lib = None
 
@@ -82,6 +84,19 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     L.fef_spec_verify_at_round.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp,
                                            vp, sz, vp, vp]
     L.fef_spec_verify_at_round.restype = i32
+    L.fef_draft_sample_with_target.argtypes = [vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp, vp, sz,
+                                               vp, vp]
+    L.fef_draft_sample_with_target.restype = i32
+    L.fef_spec_verify_with_norms.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i32, f32, u64, u32, vp, vp, vp, vp,
+                                             vp, sz, vp, vp]
+    L.fef_spec_verify_with_norms.restype = i32
+    L.fef_synth_logits.argtypes = [vp, vp, i32, i32, i32, i64, i32, f32, f32, f32, f32, u64, u32, vp, vp]
+    L.fef_synth_logits.restype = i32
+    L.fef_loop_run_synthetic_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
+    L.fef_loop_run_synthetic_workspace_bytes.restype = sz
+    L.fef_loop_run_synthetic.argtypes = [i32, i32, i32, i32, i32, f32, u64, i32, i32, f32, f32, f32, f32, vp, vp, vp, vp,
+                                         vp, sz, vp, vp]
+    L.fef_loop_run_synthetic.restype = i32
     L.fef_loop_advance_round.argtypes = [vp, vp, i32, vp]
     L.fef_loop_advance_round.restype = i32
     L.fef_vp_task_bytes.argtypes = [i32]
@@ -171,7 +186,8 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
                     V: Optional[int] = None, out: Optional[VerifyResult] = None,
                     workspace: Optional[torch.Tensor] = None, stream=None, stage_events=None,
                     draft_log2_norm: Optional[torch.Tensor] = None,
-                    device_round: Optional[torch.Tensor] = None) -> VerifyResult:
+                    device_round: Optional[torch.Tensor] = None,
+                    target_log2_norm: Optional[torch.Tensor] = None) -> VerifyResult:
     """Enqueue one verification call (see ``fef_spec_verify`` in include/fef.h).
 
     With ``stage_events`` (four ``torch.cuda.Event(enable_timing=True)`` that have
@@ -179,6 +195,8 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
     ``fef_spec_verify_profiled`` and the events mark the kernel boundaries.  With
     ``draft_log2_norm`` (the ``log2_norm`` of ``fef_draft_sample``, ``[B, K]`` float64) the
     call goes through ``fef_spec_verify_with_draft_norm`` and streams the target rows only.
+    With ``target_log2_norm`` as well (from ``fef_draft_sample(..., target_logits=...)``) it goes through
+    ``fef_spec_verify_with_norms`` and streams nothing.
     With ``device_round`` (a one-element int32 CUDA tensor) the call goes through
     ``fef_spec_verify_at_round``: the step used is ``step + device_round[0]`` when the kernels run.
 
@@ -216,7 +234,16 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
             if draft_log2_norm.dtype != torch.float64 or draft_log2_norm.numel() != B * K or \
                     not draft_log2_norm.is_contiguous() or draft_log2_norm.device != dev:
                 raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_draft_norm")
-        if device_round is not None:
+        if target_log2_norm is not None:
+            if draft_log2_norm is None or target_log2_norm.dtype != torch.float64 or target_log2_norm.numel() != B * K or \
+                    not target_log2_norm.is_contiguous() or target_log2_norm.device != dev:
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_norms")
+            if device_round is not None and (device_round.dtype != torch.int32 or device_round.numel() != 1):
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_with_norms")
+            st = load().fef_spec_verify_with_norms(*args[:3], draft_log2_norm.data_ptr(), target_log2_norm.data_ptr(),
+                                                   *args[3:12], None if device_round is None else device_round.data_ptr(),
+                                                   *args[12:])
+        elif device_round is not None:
             if device_round.dtype != torch.int32 or device_round.numel() != 1 or device_round.device != dev:
                 raise FefError(FEF_ERR_INVALID_ARG, "fef_spec_verify_at_round")
             st = load().fef_spec_verify_at_round(*args[:3], None if draft_log2_norm is None else draft_log2_norm.data_ptr(),
@@ -237,6 +264,7 @@ class DraftResult(NamedTuple):
     tokens: torch.Tensor         # [B, K] int32, -1 where nothing was drawn
     log2_norm: torch.Tensor      # [B, K] float64
     device_status: torch.Tensor  # [1] int32 (read it after synchronising)
+    target_log2_norm: Optional[torch.Tensor] = None  # [B, K] float64, when the target logits were given
 
 
 def fef_draft_sample_workspace_bytes(B: int, K: int, V: int, dtype) -> int:
@@ -247,8 +275,11 @@ def fef_draft_sample_workspace_bytes(B: int, K: int, V: int, dtype) -> int:
 def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, step: int,
                      row_len: Optional[torch.Tensor] = None, V: Optional[int] = None,
                      out: Optional[DraftResult] = None, workspace: Optional[torch.Tensor] = None,
-                     stream=None, device_round: Optional[torch.Tensor] = None) -> DraftResult:
-    """Enqueue the draft-token draws of one call (see ``fef_draft_sample`` in include/fef.h).
+                     stream=None, device_round: Optional[torch.Tensor] = None,
+                     target_logits: Optional[torch.Tensor] = None) -> DraftResult:
+    """Enqueue the draft-token draws of one call (see ``fef_draft_sample`` in include/fef.h).  With
+    ``target_logits`` (same shape and dtype) the call goes through ``fef_draft_sample_with_target`` and
+    the result also carries the target laws' normalisers.
 
     ``draft_logits``: ``[B, K, ld]`` CUDA tensor, float32 or bfloat16, contiguous; ``V`` (default
     ``ld``) entries of each row are used.  Asynchronous on the current (or given) stream.
@@ -274,7 +305,21 @@ def fef_draft_sample(draft_logits: torch.Tensor, temperature: float, seed: int, 
                 float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF)
         tail = (out.tokens.data_ptr(), out.log2_norm.data_ptr(), workspace.data_ptr(), workspace.numel(),
                 out.device_status.data_ptr(), _stream_ptr(stream))
-        if device_round is None:
+        if target_logits is not None:
+            _require_cuda(target_logits)
+            if target_logits.shape != draft_logits.shape or target_logits.dtype != draft_logits.dtype or \
+                    not target_logits.is_contiguous():
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_draft_sample_with_target")
+            tnorm = out.target_log2_norm
+            if tnorm is None:
+                tnorm = torch.empty((B, K), dtype=torch.float64, device=dev)
+                out = DraftResult(out.tokens, out.log2_norm, out.device_status, tnorm)
+            if device_round is not None and (device_round.dtype != torch.int32 or device_round.numel() != 1):
+                raise FefError(FEF_ERR_INVALID_ARG, "fef_draft_sample_with_target")
+            st = load().fef_draft_sample_with_target(head[0], target_logits.data_ptr(), *head[1:],
+                                                     None if device_round is None else device_round.data_ptr(),
+                                                     tail[0], tail[1], tnorm.data_ptr(), *tail[2:])
+        elif device_round is None:
             st = load().fef_draft_sample(*head, *tail)
         else:
             if device_round.dtype != torch.int32 or device_round.numel() != 1 or device_round.device != dev:
@@ -578,3 +623,49 @@ def fef_lmhead_logits(hidden: torch.Tensor, weight: torch.Tensor, out: Optional[
     if st != FEF_OK:
         raise FefError(st, "fef_lmhead_logits")
     return out, status
+
+
+# ---------------------------------------------------------------- device-made logits, whole loop ----
+def fef_synth_logits(B: int, K: int, V: int, dtype, draft_std: float, noise_std: float, seed: int, round: int,
+                     boost_fraction: float = 0.0, boost: float = 0.0, device_round: Optional[torch.Tensor] = None,
+                     out=None, stream=None, device="cuda"):
+    """Seeded synthetic (draft_logits, target_logits), ``[B, K, ld]`` with ``ld`` = V rounded up to whole
+    16-byte vectors (see ``fef_synth_logits`` in include/fef.h); pass ``V=V`` to the calls that read them."""
+    code = FEF_F32 if dtype == torch.float32 else FEF_BF16
+    per_vec = 4 if code == FEF_F32 else 8
+    ld = (V + per_vec - 1) // per_vec * per_vec
+    dev = torch.device(device)
+    with _on(dev, stream):
+        if out is None:
+            out = (torch.empty((B, K, ld), dtype=dtype, device=dev), torch.empty((B, K, ld), dtype=dtype, device=dev))
+        st = load().fef_synth_logits(out[0].data_ptr(), out[1].data_ptr(), B, K, V, ld, code, float(draft_std),
+                                     float(noise_std), float(boost_fraction), float(boost),
+                                     int(seed) & 0xFFFFFFFFFFFFFFFF, int(round) & 0xFFFFFFFF,
+                                     None if device_round is None else device_round.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_synth_logits")
+    return out
+
+
+def fef_loop_run_synthetic(B: int, L: int, K: int, V: int, dtype, temperature: float, seed: int, n_steps: int,
+                           remask_k: int, draft_std: float, noise_std: float, boost_fraction: float = 0.0,
+                           boost: float = 0.0, stream=None, device="cuda"):
+    """The whole decoding loop on synthetic logits as one graph launch (see ``fef_loop_run_synthetic`` in
+    include/fef.h), from an all-masked state.  Returns dict(tokens, conf, in_step, rounds, device_status)."""
+    code = FEF_F32 if dtype == torch.float32 else FEF_BF16
+    dev = torch.device(device)
+    with _on(dev, stream):
+        tokens = torch.full((B, L), MASK_TOKEN, dtype=torch.int32, device=dev)
+        conf = torch.full((B, L), -1.0, dtype=torch.float32, device=dev)
+        in_step = torch.zeros((B, L), dtype=torch.uint8, device=dev)
+        rnd = torch.zeros(1, dtype=torch.int32, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        ws = torch.empty(max(int(load().fef_loop_run_synthetic_workspace_bytes(B, L, K, V, code, remask_k)), 256),
+                         dtype=torch.uint8, device=dev)
+        st = load().fef_loop_run_synthetic(B, L, K, V, code, float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, n_steps,
+                                           remask_k, float(draft_std), float(noise_std), float(boost_fraction),
+                                           float(boost), tokens.data_ptr(), conf.data_ptr(), in_step.data_ptr(),
+                                           rnd.data_ptr(), ws.data_ptr(), ws.numel(), status.data_ptr(), _stream_ptr(stream))
+    if st != FEF_OK:
+        raise FefError(st, "fef_loop_run_synthetic")
+    return dict(tokens=tokens, conf=conf, in_step=in_step, rounds=int(rnd.item()), device_status=int(status.item()))

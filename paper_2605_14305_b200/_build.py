@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libfef.so")
-SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu", "fef_loop.cu", "fef_lmhead.cu"]
+SOURCES = ["fef_verify.cu", "fef_remask.cu", "fef_draft.cu", "fef_loop.cu", "fef_lmhead.cu", "fef_synth.cu"]
 HEADERS = [os.path.join(CSRC, h) for h in ("fef_common.cuh", "fef_device_math.cuh", "fef_verify_params.cuh",
                                             "fef_residual.cuh")] + [os.path.join(INCLUDE, "fef.h")]
 

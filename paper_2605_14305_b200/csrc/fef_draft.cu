@@ -20,7 +20,6 @@
 namespace fef {
 
 constexpr int kDraftThreads = 256;
-constexpr int kDraftBatch = 4;          // vectors a thread has in flight
 constexpr int kDraftMaxParts = 64;      // CTAs per row at most (the last one looks at 2 keys per part)
 constexpr uint32_t kStreamDraft = 2u;   // Philox stream of the draft draws
 constexpr float kKeyBand = 1.0f / 1024.0f;  // binary32 keys this close to the best one are re-scored exactly
@@ -29,11 +28,12 @@ struct __align__(16) DraftPart {  // what one CTA leaves for the row's last CTA
     float ref, sum;   // sum of 2^(l c - ref) over the part (NaN when the data is bad)
     float k1, k2;     // best two keys (-inf when empty)
     int x1, x2;       // their vocabulary ids
-    int pad[2];
+    float tref, tsum; // the same sum over the target row's part, when the call also reduces the target rows
 };
 
 struct DraftParams {
     const char* logits;
+    const char* target;  // target logits of the same shape, or null: their rows are summed in the same pass
     const int32_t* row_len;
     int B, K, V;
     int vec_elems;       // elements covered by whole 16-byte vectors; the rest is the row's tail
@@ -46,6 +46,7 @@ struct DraftParams {
     PhiloxKeys keys;     // round keys of `seed`
     int32_t* tokens;     // [B, K]
     double* log2_norm;   // [B, K] or null
+    double* target_log2_norm;  // [B, K]: log2 normaliser of the target law (with `target`)
     DraftPart* part_out; // [B*K][parts]
     unsigned* arrivals;  // [B*K], cleared by the host call
     int32_t* status;
@@ -85,6 +86,27 @@ __device__ __forceinline__ uint32_t step_of(const DraftParams& P) {
     return P.step + (P.round ? __ldg(P.round) : 0u);
 }
 
+// Rare path of the draft pass, out of line so that the loop around it stays small: the id's key
+// l c - log2(-ln u) in binary32, offered to the thread's best two and to the CTA's shared record of
+// its largest keys (two slots updated with atomic maxima, the smaller of (new, old) moving on to the
+// second slot, so a value sits in one place only and the slots hold keys of different ids).
+static __device__ __noinline__ BestTwo offer_key(BestTwo top, float lc, uint32_t word, int x, int* best2) {
+    const float key = lc - lg2_approx(neg_log_uniform(one_minus_uniform(word)));
+    top.offer(key, x);
+    int v = float_order(key);
+    if (v > *reinterpret_cast<volatile int*>(best2 + 1)) {
+        const int old = atomicMax(best2, v);
+        v = min(v, old);
+        atomicMax(best2 + 1, v);
+    }
+    return top;
+}
+// The lower bound of the CTA's second-best key that the shared record gives.
+__device__ __forceinline__ float shared_floor2(const int* best2) {
+    const volatile int* b = best2;
+    return float_unorder(min(b[0], b[1]));
+}
+
 // Exact (double) key l / T - ln(-ln u) of vocabulary id x, in units of log2: l c - log2(-ln u).
 template <int DT>
 __device__ double exact_key(int x, const char* row, double c, uint32_t b, uint32_t pos, const DraftParams& P) {
@@ -97,8 +119,8 @@ __device__ double exact_key(int x, const char* row, double c, uint32_t b, uint32
     return l * c - log2(-log(u));
 }
 
-template <int DT, bool GREEDY>
-__global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_constant__ DraftParams P) {
+template <int DT, bool GREEDY, bool WITH_TARGET>
+__global__ void __launch_bounds__(kDraftThreads, WITH_TARGET ? 3 : 4) draft_kernel(const __grid_constant__ DraftParams P) {
     constexpr int N = Elem<DT>::kPerVec;
     const int parts = P.parts;
     const int64_t row = blockIdx.x / parts;
@@ -109,108 +131,134 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
         if (part == 0 && threadIdx.x == 0) {
             P.tokens[row] = -1;
             if (P.log2_norm) P.log2_norm[row] = 0.0;
+            if (WITH_TARGET) P.target_log2_norm[row] = 0.0;
         }
         return;
     }
     const char* lrow = P.logits + row * P.ld_bytes;
+    const char* trow = WITH_TARGET ? P.target + row * P.ld_bytes : nullptr;
     const uint32_t ub = static_cast<uint32_t>(b), upos = static_cast<uint32_t>(i);
     PhiloxRow rng;
     rng.prepare(P.keys, ub, upos, step_of(P));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-    RowState st;
+    RowState st, stt;  // stt: the target row's sum (WITH_TARGET)
     st.reset();
+    stt.reset();
     BestTwo top;
     top.clear();
-    // A lower bound of the CTA's second-best key so far, as an ordered integer; a stale value is
-    // only less sharp.
-    __shared__ int s_floor;
-    if (threadIdx.x == 0) s_floor = float_order(-INFINITY);
+    // Two of the largest keys any thread of the CTA has offered so far (ordered integers, see
+    // offer_key): their minimum is a lower bound of the CTA's second-best key, the floor below which
+    // an id cannot matter.  A stale value is only less sharp.
+    __shared__ int s_best2[2];
+    if (threadIdx.x == 0) s_best2[0] = s_best2[1] = float_order(-INFINITY);
     __syncthreads();
     float floor_k = -INFINITY;
 
     const int nvec = P.vec_elems / N;
     const int v_begin = static_cast<int>(static_cast<int64_t>(part) * nvec / parts);
     const int v_end = static_cast<int>(static_cast<int64_t>(part + 1) * nvec / parts);
-    bool first = true;
-    for (int v0 = v_begin; v0 < v_end; v0 += kDraftThreads * kDraftBatch) {
-        uint4 w[kDraftBatch];
-        int vec[kDraftBatch];
+    // a lane beyond the end works on -inf logits (they never qualify), so the warp stays whole
+    constexpr uint32_t kMinusInf = DT == FEF_F32 ? 0xFF800000u : 0xFF80FF80u;
+    auto fetch = [&](int v0, uint4& w) {
+        const int vec = v0 + static_cast<int>(threadIdx.x);
+        w = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
+        if (vec < v_end) w = ld_global_nc_v4(lrow + static_cast<int64_t>(vec) * 16);
+    };
+    // One vector per thread and step, the loads of the next two steps in flight; the loop body is kept
+    // small (one copy, the rare path out of line): a larger one stalls on instruction fetch.
+    auto fetch_target = [&](int v0, uint4& w) {
+        const int vec = v0 + static_cast<int>(threadIdx.x);
+        w = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
+        if (vec < v_end) w = ld_global_nc_v4(trow + static_cast<int64_t>(vec) * 16);
+    };
+    uint4 w0, w1, w2;
+    uint4 t0, t1, t2;
+    fetch(v_begin, w0);
+    fetch(v_begin + kDraftThreads, w1);
+    if constexpr (WITH_TARGET) {
+        fetch_target(v_begin, t0);
+        fetch_target(v_begin + kDraftThreads, t1);
+    }
+#pragma unroll 1
+    for (int v0 = v_begin; v0 < v_end; v0 += kDraftThreads) {
+        fetch(v0 + 2 * kDraftThreads, w2);
+        if constexpr (WITH_TARGET) {
+            // the target row's share of the same pass: sum of 2^(l c - ref), as in the streaming kernel
+            fetch_target(v0 + 2 * kDraftThreads, t2);
+            if (v0 + static_cast<int>(threadIdx.x) < v_end) {
+                if (stt.ref == kNoReference) stt.ref = first_reference<DT>(t0, P.c_hi, P.c_lo);
+                float lt[N];
+                unpack<DT>(t0, lt);
+                float ts = 0.f;
 #pragma unroll
-        for (int j = 0; j < kDraftBatch; ++j) {
-            vec[j] = v0 + j * kDraftThreads + static_cast<int>(threadIdx.x);
-            // a lane beyond the end works on -inf logits (they never qualify), so the warp stays whole
-            constexpr uint32_t kMinusInf = DT == FEF_F32 ? 0xFF800000u : 0xFF80FF80u;
-            w[j] = make_uint4(kMinusInf, kMinusInf, kMinusInf, kMinusInf);
-            if (vec[j] < v_end) w[j] = ld_global_nc_v4(lrow + static_cast<int64_t>(vec[j]) * 16);
+                for (int t = 0; t < N; ++t) ts += exp2_scaled<DT>(lt[t], P.c_hi, P.c_lo, stt.ref);
+                if (ts <= kRescaleAbove)
+                    stt.sum += ts;
+                else
+                    absorb_vector<DT, false>(t0, 0, P.c_hi, P.c_lo, stt);
+            }
+            t0 = t1;
+            t1 = t2;
         }
-        floor_k = fmaxf(floor_k, float_unorder(*reinterpret_cast<volatile int*>(&s_floor)));
+        const int vec = v0 + static_cast<int>(threadIdx.x);
+        floor_k = fmaxf(floor_k, shared_floor2(s_best2));
+        float l[N], e[N];
+        unpack<DT>(w0, l);
+        if (st.ref == kNoReference) st.ref = first_reference<DT>(w0, P.c_hi, P.c_lo);
+        const float ref_used = st.ref;  // the slow way below may move st.ref; e[] stays relative to this one
 #pragma unroll
-        for (int j = 0; j < kDraftBatch; ++j) {
-            float l[N], e[N];
-            unpack<DT>(w[j], l);
-            if (st.ref == kNoReference) st.ref = first_reference<DT>(w[j], P.c_hi, P.c_lo);
-            const float ref_used = st.ref;  // the slow way below may move st.ref; e[] stays relative to this one
+        for (int t = 0; t < N; ++t) e[t] = exp2_scaled<DT>(l[t], P.c_hi, P.c_lo, ref_used);
+        float vs;
+        if constexpr (N == 8)
+            vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+        else
+            vs = (e[0] + e[1]) + (e[2] + e[3]);
+        if (vs <= kRescaleAbove)
+            st.sum += vs;
+        else  // reference missing or far too low, or bad data: the slow way moves it
+            absorb_vector<DT, false>(w0, 0, P.c_hi, P.c_lo, st);
+        if constexpr (GREEDY) {
+            // temperature 0: the key is the logit itself
 #pragma unroll
-            for (int t = 0; t < N; ++t) e[t] = exp2_scaled<DT>(l[t], P.c_hi, P.c_lo, ref_used);
-            float vs;
-            if constexpr (N == 8)
-                vs = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-            else
-                vs = (e[0] + e[1]) + (e[2] + e[3]);
-            if (vs <= kRescaleAbove)
-                st.sum += vs;
-            else  // reference missing or far too low, or bad data: the slow way moves it
-                absorb_vector<DT, false>(w[j], 0, P.c_hi, P.c_lo, st);
-            if constexpr (GREEDY) {
-                // temperature 0: the key is the logit itself
+            for (int t = 0; t < N; ++t)
+                if (l[t] > top.k2) top.offer(l[t], vec * N + t);
+        } else {
+            // an id can reach the floor only if 1 - u < 2^(l c - floor) = e * 2^(ref - floor)
+            // (the factor keeps an id whose key ties the floor within binary32 rounding).
+            // 1 - u < e * scale, with u's 23 bits = word >> 9, reads word > 2^32 - 256 - e * scale * 2^32:
+            // one multiply-add, one conversion (negative and NaN give 0) and one integer compare per
+            // id.  The constant 2^32 - 1024 and the factor leave room for every rounding, so no id
+            // is missed; an id let through in error (-inf logits while there is no floor yet, one
+            // word in 2^22 otherwise) is sorted out by the exact arithmetic at the end.
+            const float s32 = 1.00001f * ex2_approx(ref_used - floor_k) * 4294967296.0f * 1.00002f;
+            uint32_t word[N];
+#pragma unroll
+            for (int g4 = 0; g4 < N / 4; ++g4) {
+                const uint4 r = rng.draw(P.keys, (kStreamDraft << 30) | (static_cast<uint32_t>(vec * N + 4 * g4) >> 2));
+                word[4 * g4] = r.x;
+                word[4 * g4 + 1] = r.y;
+                word[4 * g4 + 2] = r.z;
+                word[4 * g4 + 3] = r.w;
+            }
+            unsigned qualify = 0u;
+#pragma unroll
+            for (int t = 0; t < N; ++t)
+                qualify |= (word[t] >= __float2uint_rz(fmaf(-e[t], s32, 4294966272.0f))) ? (1u << t) : 0u;
+            if (__any_sync(0xFFFFFFFFu, qualify != 0u)) {  // the vote keeps this out of the straight line
 #pragma unroll
                 for (int t = 0; t < N; ++t)
-                    if (l[t] > top.k2) top.offer(l[t], vec[j] * N + t);
-            } else {
-                // an id can reach the floor only if 1 - u < 2^(l c - floor) = e * 2^(ref - floor)
-                // (the factor keeps an id whose key ties the floor within binary32 rounding)
-                const float scale = 1.00001f * ex2_approx(ref_used - floor_k);
-#pragma unroll
-                for (int g4 = 0; g4 < N / 4; ++g4) {
-                    const int x0 = vec[j] * N + 4 * g4;
-                    const uint4 r = rng.draw(P.keys, (kStreamDraft << 30) | (static_cast<uint32_t>(x0) >> 2));
-                    // 1 - u < e * scale, with u's 23 bits = word >> 9, reads word > 2^32 - 256 - e * scale * 2^32:
-                    // one multiply-add, one conversion (negative and NaN give 0) and one integer compare per
-                    // id.  The constant 2^32 - 1024 and the factor leave room for every rounding, so no id
-                    // is missed; an id let through in error (-inf logits while there is no floor yet, one
-                    // word in 2^22 otherwise) is sorted out by the exact arithmetic below.
-                    const float s32 = scale * 4294967296.0f * 1.00002f;
-                    const bool q0 = r.x >= __float2uint_rz(fmaf(-e[4 * g4], s32, 4294966272.0f));
-                    const bool q1 = r.y >= __float2uint_rz(fmaf(-e[4 * g4 + 1], s32, 4294966272.0f));
-                    const bool q2 = r.z >= __float2uint_rz(fmaf(-e[4 * g4 + 2], s32, 4294966272.0f));
-                    const bool q3 = r.w >= __float2uint_rz(fmaf(-e[4 * g4 + 3], s32, 4294966272.0f));
-                    if (__any_sync(0xFFFFFFFFu, q0 || q1 || q2 || q3)) {  // the vote keeps this out of the straight line
-                        const float ts[4] = {one_minus_uniform(r.x), one_minus_uniform(r.y), one_minus_uniform(r.z),
-                                             one_minus_uniform(r.w)};
-                        const bool qs[4] = {q0, q1, q2, q3};
-#pragma unroll
-                        for (int t = 0; t < 4; ++t)
-                            if (qs[t] && l[4 * g4 + t] > -INFINITY) {
-                                const float lv = l[4 * g4 + t];
-                                float lc = lv * P.c_hi;
-                                if constexpr (Elem<DT>::kSplitScale) lc = fmaf(lv, P.c_lo, lc);
-                                top.offer(lc - lg2_approx(neg_log_uniform(ts[t])), x0 + t);
-                            }
+                    if ((qualify & (1u << t)) && l[t] > -INFINITY) {
+                        float lc = l[t] * P.c_hi;
+                        if constexpr (Elem<DT>::kSplitScale) lc = fmaf(l[t], P.c_lo, lc);
+                        top = offer_key(top, lc, word[t], vec * N + t, s_best2);
                     }
-                }
-            }
-            // raise the floor: any lane's second-best key bounds the CTA's second best from below
-            floor_k = fmaxf(floor_k, float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(top.k2))));
-            if (j == 0 && first) {
-                // after the first vector of every thread the whole CTA shares what it has found
-                if (lane == 0) atomicMax(&s_floor, float_order(floor_k));
-                __syncthreads();
-                floor_k = fmaxf(floor_k, float_unorder(*reinterpret_cast<volatile int*>(&s_floor)));
+                __syncwarp();
+                floor_k = fmaxf(floor_k, shared_floor2(s_best2));
             }
         }
-        first = false;
-        if (lane == 0) atomicMax(&s_floor, float_order(floor_k));
+        w0 = w1;
+        w1 = w2;
     }
 
     // ---- CTA-wide: sum and best two
@@ -218,6 +266,13 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
     float ssum = st.sum * ex2_approx(st.ref - M);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xFFFFFFFFu, ssum, o);
+    float tM = 0.f, tsum = 0.f;
+    if constexpr (WITH_TARGET) {
+        tM = float_unorder(__reduce_max_sync(0xFFFFFFFFu, float_order(stt.ref)));
+        tsum = stt.sum * ex2_approx(stt.ref - tM);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tsum += __shfl_xor_sync(0xFFFFFFFFu, tsum, o);
+    }
     top.warp_merge();
     __shared__ DraftPart s_part[kDraftThreads / 32];
     __shared__ int s_last;
@@ -229,6 +284,8 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
         d.k2 = top.k2;
         d.x1 = top.x1;
         d.x2 = top.x2;
+        d.tref = tM;
+        d.tsum = tsum;
         s_part[warp] = d;
     }
     __syncthreads();
@@ -244,6 +301,11 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
             const float Mn = fmaxf(all.ref, o.ref);
             all.sum = all.sum * ex2_approx(all.ref - Mn) + o.sum * ex2_approx(o.ref - Mn);
             all.ref = Mn;
+            if constexpr (WITH_TARGET) {
+                const float Tn = fmaxf(all.tref, o.tref);
+                all.tsum = all.tsum * ex2_approx(all.tref - Tn) + o.tsum * ex2_approx(o.tref - Tn);
+                all.tref = Tn;
+            }
             bt.offer(o.k1, o.x1);
             bt.offer(o.k2, o.x2);
         }
@@ -337,6 +399,43 @@ __global__ void __launch_bounds__(kDraftThreads, 4) draft_kernel(const __grid_co
             Z = oz;
         }
     }
+    if constexpr (WITH_TARGET) {
+        // the target law's normaliser from the parts' sums and the row's tail elements (NaN on bad data:
+        // the verification that takes it reports the window)
+        double tm = -INFINITY, ts = 0.0;
+        int tbad = 0;
+        for (int p = lane; p < parts; p += 32) {
+            const float pref = po[p].tref, psum = po[p].tsum;
+            if (!(psum >= 0.f) || psum == INFINITY) tbad = 1;
+            if (psum > 0.f) {
+                const double pm = pref, ps = psum;
+                if (pm > tm) {
+                    ts = tm > -INFINITY ? ts * exp2(tm - pm) + ps : ps;
+                    tm = pm;
+                } else {
+                    ts += ps * exp2(pm - tm);
+                }
+            }
+        }
+        for (int x = P.vec_elems + lane; x < P.V; x += 32) {
+            const float l = load_logit<DT>(trow, x);
+            if (l != l || l == INFINITY) {
+                tbad = 1;
+            } else if (l > -INFINITY) {
+                const double pm = static_cast<double>(l) * c;
+                if (pm > tm) {
+                    ts = tm > -INFINITY ? ts * exp2(tm - pm) + 1.0 : 1.0;
+                    tm = pm;
+                } else {
+                    ts += exp2(pm - tm);
+                }
+            }
+        }
+        const double tMw = warp_max(tm);
+        const double tS = warp_sum(tm > -INFINITY ? ts * exp2(tm - tMw) : 0.0);
+        tbad = __any_sync(0xFFFFFFFFu, tbad) || !(tS > 0.0) || !(tS < INFINITY);
+        if (lane == 0) P.target_log2_norm[row] = tbad ? __longlong_as_double(0x7FF8000000000000ll) : tMw + log2(tS);
+    }
     if (lane == 0) {
         const bool ok = !bad && score > -INFINITY;
         P.tokens[row] = ok ? Z : -1;
@@ -372,10 +471,19 @@ size_t fef_draft_sample_workspace_bytes(int B, int K, int V, fef_dtype dt) {
 
 }  // extern "C"
 
+template <int DT, bool GREEDY>
+static void launch_draft(const fef::DraftParams& P, unsigned grid, cudaStream_t stream) {
+    if (P.target)
+        fef::draft_kernel<DT, GREEDY, true><<<grid, fef::kDraftThreads, 0, stream>>>(P);
+    else
+        fef::draft_kernel<DT, GREEDY, false><<<grid, fef::kDraftThreads, 0, stream>>>(P);
+}
+
 static fef_status draft_impl(const void* draft_logits, const int32_t* row_len, int B, int K, int V, int64_t ld,
                              fef_dtype dt, float temperature, uint64_t seed, uint32_t step,
                              const uint32_t* device_round, int32_t* draft_tokens, double* log2_norm, void* workspace,
-                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream,
+                             const void* target_logits = nullptr, double* target_log2_norm = nullptr) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !draft_tokens) return FEF_ERR_INVALID_ARG;
@@ -384,6 +492,8 @@ static fef_status draft_impl(const void* draft_logits, const int32_t* row_len, i
     const int esize = dt == FEF_F32 ? 4 : 2;
     if (static_cast<int64_t>(V) * esize > (1ll << 30)) return FEF_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(draft_logits) & 15) || ((ld * esize) & 15)) return FEF_ERR_ALIGNMENT;
+    if (target_logits && (reinterpret_cast<uintptr_t>(target_logits) & 15)) return FEF_ERR_ALIGNMENT;
+    if ((target_logits != nullptr) != (target_log2_norm != nullptr)) return FEF_ERR_INVALID_ARG;
     int dev = -1, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
@@ -394,6 +504,8 @@ static fef_status draft_impl(const void* draft_logits, const int32_t* row_len, i
     const bool greedy = temperature == 0.0f;
     DraftParams P;
     P.logits = static_cast<const char*>(draft_logits);
+    P.target = static_cast<const char*>(target_logits);
+    P.target_log2_norm = target_log2_norm;
     P.row_len = row_len;
     P.B = B;
     P.K = K;
@@ -431,14 +543,14 @@ static fef_status draft_impl(const void* draft_logits, const int32_t* row_len, i
     const unsigned grid = static_cast<unsigned>(rows * P.parts);
     if (dt == FEF_F32) {
         if (greedy)
-            draft_kernel<FEF_F32, true><<<grid, kDraftThreads, 0, stream>>>(P);
+            launch_draft<FEF_F32, true>(P, grid, stream);
         else
-            draft_kernel<FEF_F32, false><<<grid, kDraftThreads, 0, stream>>>(P);
+            launch_draft<FEF_F32, false>(P, grid, stream);
     } else {
         if (greedy)
-            draft_kernel<FEF_BF16, true><<<grid, kDraftThreads, 0, stream>>>(P);
+            launch_draft<FEF_BF16, true>(P, grid, stream);
         else
-            draft_kernel<FEF_BF16, false><<<grid, kDraftThreads, 0, stream>>>(P);
+            launch_draft<FEF_BF16, false>(P, grid, stream);
     }
     return cudaGetLastError() == cudaSuccess ? FEF_OK : FEF_ERR_CUDA;
 }
@@ -461,6 +573,18 @@ fef_status fef_draft_sample_at_round(const void* draft_logits, const int32_t* ro
     if (!device_round) return FEF_ERR_INVALID_ARG;
     return draft_impl(draft_logits, row_len, B, K, V, ld, dt, temperature, seed, step, device_round, draft_tokens,
                       log2_norm, workspace, workspace_bytes, device_status, cuda_stream);
+}
+
+fef_status fef_draft_sample_with_target(const void* draft_logits, const void* target_logits, const int32_t* row_len,
+                                        int B, int K, int V, int64_t ld, fef_dtype dt, float temperature,
+                                        uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                        int32_t* draft_tokens, double* draft_log2_norm, double* target_log2_norm,
+                                        void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                        void* cuda_stream) {
+    if (!target_logits || !target_log2_norm) return FEF_ERR_INVALID_ARG;
+    return draft_impl(draft_logits, row_len, B, K, V, ld, dt, temperature, seed, step, device_round, draft_tokens,
+                      draft_log2_norm, workspace, workspace_bytes, device_status, cuda_stream, target_logits,
+                      target_log2_norm);
 }
 
 }  // extern "C"

@@ -401,7 +401,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
 // slices of a sharded vocabulary): one warp per row and tensor, four 16-byte loads per lane in
 // flight, one warp reduction per row, no shared memory.  Leaves one partial per row like the ring.
 constexpr int kRowsWarps = 8;        // rows a CTA works on at a time
-constexpr int kRowsCtasPerSm = 4;
+constexpr int kRowsCtasPerSm = 3;  // (four would cap the kernel at 64 registers: it spilled up to 412 bytes there)
 
 template <int DT, bool GREEDY>
 __global__ void __launch_bounds__(kRowsWarps * 32, kRowsCtasPerSm) rows_kernel(const __grid_constant__ VerifyParams P) {
@@ -899,7 +899,14 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_ker
     if (!wide) {
         if (my < n) {
             const int64_t row = static_cast<int64_t>(b) * G.K + my;
-            const RowNorm np = fold_unit<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P);
+            RowNorm np;
+            if (P.target_norm) {  // both laws' normalisers came with the drafts: nothing was streamed
+                np.M = P.target_norm[row];
+                np.S = 1.0;
+                np.bad = !(fabs(np.M) < INFINITY);
+            } else {
+                np = fold_unit<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P);
+            }
             RowNorm nq;
             if (P.draft_norm) {  // rho(x) = 2^(l_x c - norm): the normaliser came with the drafts
                 nq.M = P.draft_norm[row];
@@ -916,7 +923,14 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_ker
             const int i = warp + j * kResidualWarps;
             if (i >= n) break;  // uniform over the warp
             const int64_t row = static_cast<int64_t>(b) * G.K + i;
-            const RowNorm np = fold_unit_warp<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P, lane);
+            RowNorm np;
+            if (P.target_norm) {
+                np.M = P.target_norm[row];
+                np.S = 1.0;
+                np.bad = !(fabs(np.M) < INFINITY);
+            } else {
+                np = fold_unit_warp<DT, false>(row * G.units_per_row, P.target + row * G.ld_bytes, c, P, lane);
+            }
             RowNorm nq;
             if (P.draft_norm) {
                 nq.M = P.draft_norm[row];
@@ -1287,7 +1301,11 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         g_attr_done[dev][which] = true;
     }
     cudaError_t e;
-    if (events) {
+    if (!GREEDY && P.target_norm) {
+        // both laws' normalisers are given: only the counters are cleared, then the last kernel runs
+        e = launch_dependent(begin_call_kernel, dim3(1), dim3(kBeginThreads), 0, stream, P.ctl, P.tasks, G.B, P.status);
+        if (e != cudaSuccess) return e;
+    } else if (events) {
         // timing marks asked for: clear with memset nodes and launch the streaming kernel the
         // ordinary way, so that the first two marks bracket that kernel alone
         if (P.status && (e = cudaMemsetAsync(P.status, 0, sizeof(int32_t), stream)) != cudaSuccess) return e;
@@ -1377,7 +1395,7 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
                               fef_dtype dt, float temperature, uint64_t seed, uint32_t step, int32_t* accept_len,
                               int32_t* tokens, float* conf, void* workspace, size_t workspace_bytes,
                               int32_t* device_status, void* cuda_stream, void* const* stage_events,
-                              const uint32_t* device_round = nullptr) {
+                              const uint32_t* device_round = nullptr, const double* target_log2_norm = nullptr) {
     using namespace fef;
     if (dt != FEF_F32 && dt != FEF_BF16) return FEF_ERR_DTYPE;
     if (!draft_logits || !target_logits || !draft_tokens || !accept_len || !tokens || !conf)
@@ -1431,6 +1449,7 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
     P.draft_tokens = draft_tokens;
     P.row_len = row_len;
     P.draft_norm = greedy ? nullptr : draft_log2_norm;
+    P.target_norm = (greedy || !draft_log2_norm) ? nullptr : target_log2_norm;
     P.seed = seed;
     P.keys = philox_round_keys(seed);
     P.step = step;
@@ -1494,6 +1513,18 @@ fef_status fef_spec_verify_with_draft_norm(const void* draft_logits, const void*
                        cuda_stream, nullptr);
 }
 
+fef_status fef_spec_verify_with_norms(const void* draft_logits, const void* target_logits, const int32_t* draft_tokens,
+                                      const double* draft_log2_norm, const double* target_log2_norm,
+                                      const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
+                                      float temperature, uint64_t seed, uint32_t step, const uint32_t* device_round,
+                                      int32_t* accept_len, int32_t* tokens, float* conf, void* workspace,
+                                      size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    if (!draft_log2_norm || !target_log2_norm) return FEF_ERR_INVALID_ARG;
+    return verify_impl(draft_logits, target_logits, draft_tokens, row_len, draft_log2_norm, B, K, V, ld, dt,
+                       temperature, seed, step, accept_len, tokens, conf, workspace, workspace_bytes, device_status,
+                       cuda_stream, nullptr, device_round, target_log2_norm);
+}
+
 fef_status fef_spec_verify_at_round(const void* draft_logits, const void* target_logits,
                                     const int32_t* draft_tokens, const double* draft_log2_norm,
                                     const int32_t* row_len, int B, int K, int V, int64_t ld, fef_dtype dt,
@@ -1542,6 +1573,7 @@ static fef_status vp_setup(const void* draft_slice, const void* target_slice, co
     if (!(P.c_hi > 0.f) || isinf(P.c_hi)) return FEF_ERR_INVALID_ARG;
     P.wait_limit_ns = kWaitLimitNs;
     P.withhold_stage = -1;
+    P.target_norm = nullptr;
     P.target = static_cast<const char*>(target_slice);
     P.draft = static_cast<const char*>(draft_slice);
     P.draft_tokens = draft_tokens;

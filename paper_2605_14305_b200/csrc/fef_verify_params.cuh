@@ -35,6 +35,8 @@ struct VerifyParams {
     const int32_t* draft_tokens;
     const int32_t* row_len;
     const double* draft_norm;  // [B*K] log2 normalisers of the draft laws, or null: stream the draft rows
+    const double* target_norm; // [B*K] log2 normalisers of the target laws, or null (given only together with draft_norm:
+                               // then nothing is streamed)
     float c_hi, c_lo;     // log2(e)/T split in two binary32 numbers, c_lo > 0 (or 0 for bfloat16)
     double c_exact;       // log2(e)/T in double precision (the double-precision pass of the residual draw)
     unsigned long long wait_limit_ns;  // how long a wait inside the streaming kernel may last

@@ -85,7 +85,8 @@ def run_decode_loop(B: int, L: int, K: int, n_steps: int, remask_k: int,
 
 def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: int, logits_fn: Callable,
                            temperature: float, seed: int, on_round: Optional[Callable] = None,
-                           first_round: int = 0, reuse_draft_norm: bool = True, build_inputs: bool = False):
+                           first_round: int = 0, reuse_draft_norm: bool = True, build_inputs: bool = False,
+                           reuse_target_norm: bool = False, V: Optional[int] = None):
     """Algorithm 2 with the whole state resident on the device: every step of a round is one
     library call (``fef_loop_next_window`` -> [``fef_loop_verification_inputs``] ->
     ``fef_draft_sample`` -> ``fef_spec_verify`` -> ``fef_loop_commit``), and a denoising step ends
@@ -96,6 +97,9 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
     CUDA, inputs [B,K,L] int32 CUDA or None) -> (draft_logits, target_logits), both [B,K,V] CUDA.
     on_round(round, dict of the round's device tensors): optional hook, called after the commit with
     the state before it under "before"; called with round None after each re-masking.
+    reuse_target_norm: the draft draws also reduce the target rows (``fef_draft_sample(target_logits=)``)
+    and the verification takes both normalisers, so both tensors are read once per round.
+    V: vocabulary size when the logits' row pitch is larger.
 
     Returns dict(tokens [B,L] int32, conf [B,L] float32 (CUDA), rounds, committed_per_round, loop_seconds).
     """
@@ -114,12 +118,14 @@ def run_decode_loop_device(fef, B: int, L: int, K: int, n_steps: int, remask_k: 
                 break
             inputs = None
             q, p = logits_fn(rnd, window, row_len, None)
-            draft = fef.fef_draft_sample(q, temperature, seed, rnd, row_len=row_len)
+            draft = fef.fef_draft_sample(q, temperature, seed, rnd, row_len=row_len, V=V,
+                                         target_logits=p if reuse_target_norm else None)
             if build_inputs:
                 inputs = fef.fef_loop_verification_inputs(tokens, window, row_len, draft.tokens)
-            norm = draft.log2_norm if reuse_draft_norm else None
-            res = fef.fef_spec_verify(q, p, draft.tokens, temperature, seed, rnd, row_len=row_len,
-                                      draft_log2_norm=norm)
+            norm = draft.log2_norm if (reuse_draft_norm or reuse_target_norm) else None
+            res = fef.fef_spec_verify(q, p, draft.tokens, temperature, seed, rnd, row_len=row_len, V=V,
+                                      draft_log2_norm=norm,
+                                      target_log2_norm=draft.target_log2_norm if reuse_target_norm else None)
             before = (tokens.clone(), conf.clone(), in_step.clone()) if on_round is not None else None
             committed = fef.fef_loop_commit(window, row_len, res, tokens, conf, in_step)
             if on_round is not None:

@@ -197,3 +197,75 @@ def test_replayed_graph_of_a_round_equals_the_eager_device_loop(fef, B, K, L, dt
     assert g["rounds"] == a["rounds"]
     assert (g["tokens"] == a["tokens"]).all() and (g["conf"] == a["conf"]).all()
     assert (g["tokens"] >= 0).all()
+
+
+def test_device_made_logits_are_seeded_shaped_and_reproducible(fef):
+    B, K, V = 3, 5, 40000
+    for dtype in (torch.bfloat16, torch.float32):
+        q, p = fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, seed=9, round=4, boost_fraction=0.01, boost=8.0)
+        q2, p2 = fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, seed=9, round=4, boost_fraction=0.01, boost=8.0)
+        rnd = torch.tensor([3], dtype=torch.int32, device="cuda")
+        q3, p3 = fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, seed=9, round=1, boost_fraction=0.01, boost=8.0,
+                                      device_round=rnd)
+        q4, _ = fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, seed=9, round=5, boost_fraction=0.01, boost=8.0)
+        torch.cuda.synchronize()
+        assert torch.equal(q, q2) and torch.equal(p, p2) and torch.equal(q, q3) and torch.equal(p, p3)
+        assert not torch.equal(q, q4)
+        qf, pf = q[:, :, :V].float(), p[:, :, :V].float()
+        boosted = qf > 6.0                         # 2 sigma draws reach 6 with probability 1e-3; boosted ones start at 8 - 6
+        assert abs(boosted.float().mean().item() - 5 / 512) < 2e-3
+        base = torch.where(boosted, qf - 8.0, qf)
+        assert abs(base.mean().item()) < 0.02 and abs(base.std().item() - 2.0) < 0.03
+        d = pf - qf
+        assert abs(d.mean().item()) < 0.01 and abs(d.std().item() - 0.7) < 0.02
+        rows = qf.reshape(B * K, V)
+        assert abs(torch.corrcoef(torch.stack([rows[0], rows[1]]))[0, 1].item()) < 0.02   # rows are independent
+
+
+@pytest.mark.parametrize("B,K,L,dtype", [(1, 4, 40, torch.float32), (4, 8, 96, torch.bfloat16), (3, 32, 200, torch.bfloat16)])
+def test_whole_loop_as_one_graph_launch_equals_the_eager_device_loop(fef, B, K, L, dtype):
+    """fef_loop_run_synthetic (all rounds of all denoising steps as the body of a graph WHILE node, no host
+    in between) against the eager device-resident loop making the same calls round by round."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device
+
+    V, T, seed, steps, k = 3000, 1.0, 33, 3, 4
+
+    def logits_fn(rnd, window, row_len, inputs):
+        return fef.fef_synth_logits(B, K, V, dtype, 2.0, 0.7, seed, rnd, boost_fraction=0.01, boost=8.0)
+
+    a = run_decode_loop_device(fef, B, L, K, steps, k, logits_fn, T, seed, reuse_target_norm=True, V=V)
+    g = fef.fef_loop_run_synthetic(B, L, K, V, dtype, T, seed, steps, k, 2.0, 0.7, boost_fraction=0.01, boost=8.0)
+    torch.cuda.synchronize()
+    assert g["device_status"] == 0
+    assert g["rounds"] == a["rounds"]
+    assert (g["tokens"] == a["tokens"]).all() and (g["conf"] == a["conf"]).all()
+    assert (g["tokens"] >= 0).all()
+
+
+def test_eager_loop_with_both_normalisers_matches_the_oracle_round_by_round(fef):
+    """The calls the one-launch loop makes (device-made logits, draft draws that also reduce the target
+    rows, verification that takes both normalisers), checked against the oracle on every round."""
+    from paper_2605_14305_b200.decode_loop import run_decode_loop_device
+
+    B, K, L, V, T, seed = 3, 8, 64, 5000, 0.9, 17
+    st = dict(rounds=0)
+
+    def logits_fn(rnd, window, row_len, inputs):
+        return fef.fef_synth_logits(B, K, V, torch.bfloat16, 2.0, 0.7, seed, rnd, boost_fraction=0.01, boost=8.0)
+
+    def on_round(rnd, d):
+        if rnd is None:
+            return
+        orl = d["row_len"].cpu().numpy()
+        od = oracle.draft_sample(d["q"].cpu(), T, seed, rnd, row_len=orl, V=V)
+        used = np.arange(K)[None, :] < orl[:, None]
+        dt = d["draft"].tokens.cpu().numpy()
+        assert (dt[used] == od["tokens"][used]).all()
+        ref = oracle.spec_verify(d["q"].cpu(), d["p"].cpu(), dt, T, seed, rnd, row_len=orl, V=V)
+        r = d["result"]
+        rep = compare_verify(r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy(), ref)
+        assert rep.ok, rep.mismatches[:5]
+        st["rounds"] += 1
+
+    out = run_decode_loop_device(fef, B, L, K, 2, 3, logits_fn, T, seed, on_round=on_round, reuse_target_norm=True, V=V)
+    assert (out["tokens"] >= 0).all() and st["rounds"] == out["rounds"]

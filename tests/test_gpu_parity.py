@@ -370,3 +370,52 @@ def test_verification_with_the_draft_normalisers_streams_the_target_only(fef):
     torch.cuda.synchronize()
     assert int(r.device_status.item()) == fef.FEF_ERR_NONFINITE
     assert r.accept_len[1].item() == -1 and (r.accept_len[[0, 2]] == plain.accept_len[[0, 2]]).all()
+
+
+def test_draft_draws_with_the_target_normalisers_and_verification_without_streaming(fef):
+    """fef_draft_sample(target_logits=...) -> fef_spec_verify(draft_log2_norm=, target_log2_norm=):
+    both tensors are read once, by the draft kernel; the pair equals the oracle pair and the plain calls."""
+    total = ParityReport()
+    for w, T, seed in ((synth.LLADA_BATCHED.with_(B=5, K=16), 0.7, 51), (synth.LLADA_SINGLE.with_(K=8), 1.0, 52),
+                       (synth.TINY.with_(B=90, K=32, V=3001, dtype=torch.bfloat16), 1.0, 54),
+                       (synth.TINY.with_(B=3, K=5, V=37), 1.0, 55),
+                       (synth.DREAM_LARGE.with_(B=3, K=8, dtype=torch.float32), 1.0, 53)):
+        q, p = synth.make_logits(w, seed=seed, device="cuda")
+        if w.V % 8:  # rows must start on 16-byte boundaries: pad the pitch
+            ld = (w.V + 7) // 8 * 8
+            qq = torch.full((w.B, w.K, ld), float("nan"), dtype=q.dtype, device="cuda")
+            pp = torch.full((w.B, w.K, ld), float("nan"), dtype=q.dtype, device="cuda")
+            qq[:, :, :w.V], pp[:, :, :w.V] = q, p
+            q, p = qq, pp
+        rl = torch.randint(0, w.K + 1, (w.B,), dtype=torch.int32, device="cuda") if w.B > 2 else None
+        d = fef.fef_draft_sample(q, T, seed, 7, row_len=rl, V=w.V, target_logits=p)
+        plain_d = fef.fef_draft_sample(q, T, seed, 7, row_len=rl, V=w.V)
+        r = fef.fef_spec_verify(q, p, d.tokens, T, seed, 7, row_len=rl, V=w.V, draft_log2_norm=d.log2_norm,
+                                target_log2_norm=d.target_log2_norm)
+        plain = fef.fef_spec_verify(q, p, d.tokens, T, seed, 7, row_len=rl, V=w.V)
+        torch.cuda.synchronize()
+        assert int(r.device_status.item()) == 0 and int(d.device_status.item()) == 0
+        assert (d.tokens == plain_d.tokens).all() and (d.log2_norm == plain_d.log2_norm).all()
+        n = np.full(w.B, w.K) if rl is None else rl.cpu().numpy()
+        used = np.arange(w.K)[None, :] < n[:, None]
+        want = torch.logsumexp(p.cpu()[..., :w.V].double() / float(np.float32(T)), dim=-1).numpy() / math.log(2.0)
+        assert np.allclose(d.target_log2_norm.cpu().numpy()[used], want[used], rtol=0, atol=2e-5)
+        assert (d.target_log2_norm.cpu().numpy()[~used] == 0).all()
+        ref = oracle.spec_verify(q.cpu(), p.cpu(), d.tokens.cpu(), T, seed, 7, row_len=None if rl is None else rl.cpu(),
+                                 V=w.V)
+        rep = compare_verify(r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy(), ref)
+        assert rep.ok, rep.mismatches[:5]
+        total.merge(rep)
+        assert (r.accept_len == plain.accept_len).all() and (r.tokens == plain.tokens).all()
+        assert torch.allclose(r.conf, plain.conf, rtol=1e-5, atol=0)
+    assert total.within_budget
+    # a target row with bad data poisons its window only; temperature 0 ignores the normalisers
+    pb = p.clone()
+    pb[1, 0, 5] = float("nan")
+    d2 = fef.fef_draft_sample(q, T, seed, 7, target_logits=pb)
+    r2 = fef.fef_spec_verify(q, pb, d2.tokens, T, seed, 7, draft_log2_norm=d2.log2_norm, target_log2_norm=d2.target_log2_norm)
+    g0 = fef.fef_spec_verify(q, p, d.tokens, 0.0, seed, 7, draft_log2_norm=d.log2_norm, target_log2_norm=d.target_log2_norm)
+    g1 = fef.fef_spec_verify(q, p, d.tokens, 0.0, seed, 7)
+    torch.cuda.synchronize()
+    assert int(r2.device_status.item()) == fef.FEF_ERR_NONFINITE and int(r2.accept_len[1].item()) == -1
+    assert (g0.tokens == g1.tokens).all() and (g0.conf == g1.conf).all()

@@ -5,8 +5,9 @@ inside a memory plan that someone else owns (a server that carved up the whole d
 start-up), or on a path where an allocation's implicit synchronisation is unacceptable.
 For them the scratch lives in a fixed array inside the library.  This test drives that
 entry point through the C ABI twice in a row on different inputs and sizes and checks
-each result against fef_spec_verify with a caller-provided workspace: the integers must
-be identical and the confidences must agree to the tolerance the other GPU tests use.
+each result against fef_spec_verify with a caller-provided workspace (the integers must
+be identical and the confidences must agree to the tolerance the other GPU tests use)
+and, directly, against the CPU oracle.
 The second call also shows that what the first call left in the shared scratch does not
 leak into later results.  Collected last on purpose (file name), so a run that stops at
 the first failure has already run every other test.
@@ -27,6 +28,15 @@ def _case(B, K, V, dtype, seed):
     return synth.make_call(w, seed=seed, device="cuda")
 
 
+def _matches_oracle(got, q, p, tok, T, seed, step, row_len=None):
+    import oracle
+    from oracle.compare import compare_verify
+
+    ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), T, seed, step, row_len=None if row_len is None else row_len.cpu())
+    rep = compare_verify(got.accept_len.cpu().numpy(), got.tokens.cpu().numpy(), got.conf.cpu().numpy(), ref)
+    assert rep.ok and rep.excused == 0, rep.mismatches[:5]
+
+
 def _same(a, b):
     assert (a.accept_len.cpu().numpy() == b.accept_len.cpu().numpy()).all()
     assert (a.tokens.cpu().numpy() == b.tokens.cpu().numpy()).all()
@@ -45,6 +55,7 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice_in_a_row
     got = fef.fef_spec_verify_static(q, p, tok, 0.7, seed=5, step=1)
     torch.cuda.synchronize()
     _same(got, want)
+    _matches_oracle(got, q, p, tok, 0.7, 5, 1)
     assert (want.accept_len.cpu().numpy() < 32).any()  # the residual path ran
 
     # second call right after it: other sizes, other dtype, a ragged row length, fewer windows,
@@ -55,12 +66,14 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice_in_a_row
     got = fef.fef_spec_verify_static(q, p, tok, 1.0, seed=6, step=2, row_len=row_len)
     torch.cuda.synchronize()
     _same(got, want)
+    _matches_oracle(got, q, p, tok, 1.0, 6, 2, row_len=row_len)
 
     # and the greedy mode through the same scratch
     want = fef.fef_spec_verify(q, p, tok, 0.0, seed=6, step=3)
     got = fef.fef_spec_verify_static(q, p, tok, 0.0, seed=6, step=3)
     torch.cuda.synchronize()
     _same(got, want)
+    _matches_oracle(got, q, p, tok, 0.0, 6, 3)
 
 
 def test_static_scratch_entry_point_refuses_sizes_beyond_its_buffer():

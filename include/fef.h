@@ -108,7 +108,13 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt);
  *   device_status    device out, [1] int32, or NULL.  Set to FEF_OK at the start of the call,
  *                    then to the largest device-side error.  Windows with a data error get
  *                    accept_len = -1 and no committed tokens; other windows are unaffected.
+ *                    FEF_ERR_TIMEOUT (a bounded wait inside the streaming kernel ran out, which only
+ *                    a fault elsewhere on the device can cause): no window is decided, every
+ *                    accept_len is -1.
  *   cuda_stream      stream to enqueue on
+ *
+ * Calls that stream little (few rows) use kernels built for latency, larger ones a streaming kernel
+ * built for bandwidth; the results are the same up to the rounding order of the row sums.
  */
 fef_status fef_spec_verify(const void* draft_logits, const void* target_logits,
                            const int32_t* draft_tokens, const int32_t* row_len,

@@ -216,7 +216,9 @@ def fef_spec_verify(draft_logits: torch.Tensor, target_logits: torch.Tensor, dra
     V = ld if V is None else int(V)
     code = _dtype_code(draft_logits)
     dev = draft_logits.device
-    with _on(dev, stream):
+    # (nothing to allocate and the device already current: no context to enter, which matters for small calls)
+    plain = out is not None and workspace is not None and stream is None and torch.cuda.current_device() == dev.index
+    with (contextlib.nullcontext() if plain else _on(dev, stream)):
         if out is None:
             out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
                                torch.empty((B, K), dtype=torch.int32, device=dev),
@@ -459,7 +461,9 @@ def fef_spec_verify_static(draft_logits: torch.Tensor, target_logits: torch.Tens
     V = ld if V is None else int(V)
     code = _dtype_code(draft_logits)
     dev = draft_logits.device
-    with _on(dev, stream):
+    # (nothing to allocate and the device already current: no context to enter, which matters for small calls)
+    plain = out is not None and workspace is not None and stream is None and torch.cuda.current_device() == dev.index
+    with (contextlib.nullcontext() if plain else _on(dev, stream)):
         if out is None:
             out = VerifyResult(torch.empty(B, dtype=torch.int32, device=dev),
                                torch.empty((B, K), dtype=torch.int32, device=dev),

@@ -95,7 +95,9 @@ __device__ __forceinline__ float first_reference(const uint4& w, float c_hi, flo
     float vmax = l[0];
 #pragma unroll
     for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, l[i]);
-    return (vmax > -INFINITY && vmax < INFINITY) ? fmaf(vmax, c_lo, vmax * c_hi) : kNoReference;
+    // (rounded to an integer: two partial sums of a row are then brought to a common reference by an exact
+    // power of two, which the fold builds from the exponent instead of calling exp2)
+    return (vmax > -INFINITY && vmax < INFINITY) ? rintf(fmaf(vmax, c_lo, vmax * c_hi)) : kNoReference;
 }
 
 // Monotone map between floats without NaN and signed integers (for integer warp reductions).

@@ -426,7 +426,22 @@ __device__ void residual_draw(const VerifyParams& P, int b, int pos, double kp_d
         if (warp == 0) {
             Top3 all;
             all.clear();
-            for (int j = lane; j < ncand; j += 32) all.offer(cand[j].w, cand[j].x);
+            if constexpr (CLUSTER) {  // at most 8 x 3 candidates, in shared memory
+                for (int j = lane; j < ncand; j += 32) all.offer(cand[j].w, cand[j].x);
+            } else {
+                for (int j0 = 0; j0 < ncand; j0 += 8 * 32) {  // (all loads of a round first: they are volatile)
+                    float cw[8];
+                    int cx[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int j = j0 + k * 32 + lane;
+                        cw[k] = j < ncand ? cand[j].w : 0.f;
+                        cx[k] = j < ncand ? cand[j].x : 0x7FFFFFFF;  // (an empty slot, as Top3 keeps them)
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) all.offer(cw[k], cx[k]);
+                }
+            }
             all.warp_merge();
             // lanes 0 and 1: the ids of the two largest bounds.  First in binary32 with the same bounds as
             // the pass (a few hundred cycles); only when those do not separate them, in double precision.

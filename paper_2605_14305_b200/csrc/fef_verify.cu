@@ -472,6 +472,15 @@ struct RowNorm {
     bool data_bad; // a NaN or +inf was seen (bad also covers rows without any finite logit)
 };
 
+// 2^d for the difference d <= 0 of two reference exponents.  The streaming kernels round their references
+// to integers, so d is an integer unless a sum had to be re-referenced: then the power is assembled from its
+// exponent (exact) instead of going through exp2.
+__device__ __forceinline__ double pow2_of_difference(double d) {
+    const int n = static_cast<int>(d);
+    if (static_cast<double>(n) == d && n > -1000 && n <= 0) return __hiloint2double((1023 + n) << 20, 0);
+    return exp2(d);
+}
+
 // Fold the claims' partials of unit u (and the row's tail elements, which the streaming
 // kernel does not touch) into the row's normaliser.  One thread.
 template <int DT, bool GREEDY>
@@ -489,10 +498,10 @@ __device__ __forceinline__ RowNorm fold_unit(int64_t u, const char* row, double 
         if (p.sum > 0.f) {
             const double pm = p.ref, ps = p.sum;
             if (pm > m) {  // (the first record, and any record equal to the running reference, needs no scaling)
-                sacc = m > -INFINITY ? sacc * exp2(m - pm) + ps : ps;
+                sacc = m > -INFINITY ? sacc * pow2_of_difference(m - pm) + ps : ps;
                 m = pm;
             } else {
-                sacc += pm == m ? ps : ps * exp2(pm - m);
+                sacc += pm == m ? ps : ps * pow2_of_difference(pm - m);
             }
         }
         if (GREEDY && better(p.best, p.index, best, index)) {
@@ -642,10 +651,10 @@ __device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const Ve
         if (p.sum > 0.f) {
             const double pm = p.ref, ps = p.sum;
             if (pm > m) {  // (the first record, and any record equal to the running reference, needs no scaling)
-                sacc = m > -INFINITY ? sacc * exp2(m - pm) + ps : ps;
+                sacc = m > -INFINITY ? sacc * pow2_of_difference(m - pm) + ps : ps;
                 m = pm;
             } else {
-                sacc += pm == m ? ps : ps * exp2(pm - m);
+                sacc += pm == m ? ps : ps * pow2_of_difference(pm - m);
             }
         }
         if (GREEDY && better(p.best, p.index, best, index)) {
@@ -684,7 +693,7 @@ __device__ RowNorm fold_unit_warp(int64_t u, const char* row, double c, const Ve
             }
         }
     }
-    const double S = warp_sum(m > -INFINITY ? sacc * exp2(m - M) : 0.0);
+    const double S = warp_sum(m > -INFINITY ? sacc * pow2_of_difference(m - M) : 0.0);
     RowNorm out;
     out.M = M;
     out.S = S;
@@ -849,26 +858,19 @@ __device__ __forceinline__ int accept_test(const VerifyParams& P, int b, int i, 
     return 0;
 }
 
-template <int DT, bool CLUSTER>
-__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_kernel(const __grid_constant__ VerifyParams P) {
+// What the acceptance tests need besides the normalisers, fetched before those are waited for: the
+// draft token of "my" position and the two logits at it.  Thread form: position threadIdx.x.  Warp
+// form (wide): lane j of warp w holds position w + j * kResidualWarps.
+template <int DT>
+__device__ __forceinline__ void fetch_my_position(const VerifyParams& P, int b, int n, bool wide, int& my, int& x,
+                                                  double& lpx, double& lqx) {
     const Geometry& G = P.geo;
-    __shared__ TailShared ts;
-    __shared__ ResidualShared sh;
-    const int b = blockIdx.y, part = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
-    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
-    // very many partials per row: a warp per position shares the fold; otherwise a thread per position
-    // (with eight warps and up to 64 positions, the serial fold of a few dozen partials is still faster)
-    const bool wide = G.claims_per_unit > 32;
-
-    // what does not depend on the streaming kernel is fetched before waiting for it: the draft token
-    // of "my" position and the two logits at it.  Thread form: position threadIdx.x.  Warp form: lane j
-    // of warp w holds position w + j * kResidualWarps.
-    const int my = wide ? (lane < FEF_MAX_K / kResidualWarps ? warp + lane * kResidualWarps : FEF_MAX_K)
-                        : static_cast<int>(threadIdx.x);
-    int x = -1;
-    double lpx = 0.0, lqx = 0.0;
+    my = wide ? (lane < FEF_MAX_K / kResidualWarps ? warp + lane * kResidualWarps : FEF_MAX_K)
+              : static_cast<int>(threadIdx.x);
+    x = -1;
+    lpx = 0.0;
+    lqx = 0.0;
     if (my < n) {
         const int64_t row = static_cast<int64_t>(b) * G.K + my;
         x = __ldg(P.draft_tokens + row);
@@ -877,28 +879,25 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_ker
             lqx = load_logit<DT>(P.draft + row * G.ld_bytes, x);
         }
     }
-    if (threadIdx.x == 0) {
-        ts.rejected[0] = ts.rejected[1] = 0u;
-        ts.err = 0;
-        sh.floor_bits = sh.best3[0] = sh.best3[1] = sh.best3[2] = 0u;
-    }
-    __syncthreads();
-    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+}
 
-    if (P.ctl->aborted) {  // a wait in the streaming kernel ran out (status FEF_ERR_TIMEOUT): no window is decided
-        if (part == 0) {
-            for (int i = threadIdx.x; i < G.K; i += kResidualThreads) {
-                P.tokens[static_cast<int64_t>(b) * G.K + i] = -1;
-                P.conf[static_cast<int64_t>(b) * G.K + i] = -1.f;
-            }
-            if (threadIdx.x == 0) P.accept_len[b] = -1;
-        }
-        return;
-    }
-
+// The acceptance tests of window b from the partials (whole CTA; `ts` cleared and a barrier passed
+// before).  Returns the first rejected position (n when every draft was accepted); ts.err holds a
+// data error, if any.
+template <int DT>
+__device__ __forceinline__ int window_accept(const VerifyParams& P, int b, int n, bool wide, int my, int x, double lpx,
+                                             double lqx, double c, TailShared& ts) {
+    const Geometry& G = P.geo;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (!wide) {
         if (my < n) {
             const int64_t row = static_cast<int64_t>(b) * G.K + my;
+            if (G.claims_per_unit > 1) {
+                // several partials per row, read one after the other below: have them all on their way to L1 first
+                const Partial* recs = P.partials + row * G.units_per_row * G.claims_per_unit;
+                for (int r = 0; r < G.units_per_row * G.claims_per_unit; r += 2)
+                    asm volatile("prefetch.global.L1 [%0];" ::"l"(recs + r));
+            }
             RowNorm np;
             if (P.target_norm) {  // both laws' normalisers came with the drafts: nothing was streamed
                 np.M = P.target_norm[row];
@@ -948,30 +947,176 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_ker
         }
     }
     __syncthreads();
-
-    const int err = ts.err;
     int a = n;
     if (ts.rejected[0])
         a = __ffs(ts.rejected[0]) - 1;
     else if (ts.rejected[1])
         a = 32 + __ffs(ts.rejected[1]) - 1;
+    return a;
+}
 
-    if (part == 0) {
-        for (int i = threadIdx.x; i < G.K; i += kResidualThreads) {
-            const int64_t row = static_cast<int64_t>(b) * G.K + i;
-            const bool keep = !err && i < a;
-            P.tokens[row] = keep ? ts.tok[i] : -1;
-            P.conf[row] = keep ? ts.conf[i] : -1.f;
-        }
-        if (threadIdx.x == 0) {
-            P.accept_len[b] = err ? -1 : a;
-            if (err) report(P.status, err);
-        }
+// Window b's accepted tokens, confidences and length (one CTA of the window calls this).
+__device__ __forceinline__ void write_window(const VerifyParams& P, int b, int a, int err, const TailShared& ts) {
+    const Geometry& G = P.geo;
+    for (int i = threadIdx.x; i < G.K; i += kResidualThreads) {
+        const int64_t row = static_cast<int64_t>(b) * G.K + i;
+        const bool keep = !err && i < a;
+        P.tokens[row] = keep ? ts.tok[i] : -1;
+        P.conf[row] = keep ? ts.conf[i] : -1.f;
     }
+    if (threadIdx.x == 0) {
+        P.accept_len[b] = err ? -1 : a;
+        if (err) report(P.status, err);
+    }
+}
+// A window that stays undecided (a wait ran out).
+__device__ __forceinline__ void write_window_undecided(const VerifyParams& P, int b) {
+    const Geometry& G = P.geo;
+    for (int i = threadIdx.x; i < G.K; i += kResidualThreads) {
+        P.tokens[static_cast<int64_t>(b) * G.K + i] = -1;
+        P.conf[static_cast<int64_t>(b) * G.K + i] = -1.f;
+    }
+    if (threadIdx.x == 0) P.accept_len[b] = -1;
+}
+
+template <int DT, bool CLUSTER>
+__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) tail_kernel(const __grid_constant__ VerifyParams P) {
+    const Geometry& G = P.geo;
+    __shared__ TailShared ts;
+    __shared__ ResidualShared sh;
+    const int b = blockIdx.y, part = blockIdx.x;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    const double c = static_cast<double>(P.c_hi) + static_cast<double>(P.c_lo);
+    // very many partials per row: a warp per position shares the fold; otherwise a thread per position
+    // (with eight warps and up to 64 positions, the serial fold of a few dozen partials is still faster)
+    const bool wide = G.claims_per_unit > 32;
+
+    int my, x;
+    double lpx, lqx;
+    fetch_my_position<DT>(P, b, n, wide, my, x, lpx, lqx);
+    if (threadIdx.x == 0) {
+        ts.rejected[0] = ts.rejected[1] = 0u;
+        ts.err = 0;
+        sh.floor_bits = sh.best3[0] = sh.best3[1] = sh.best3[2] = 0u;
+    }
+    __syncthreads();
+    cudaGridDependencySynchronize();  // the streaming kernel's partials must be complete and visible
+
+    if (P.ctl->aborted) {  // a wait in the streaming kernel ran out (status FEF_ERR_TIMEOUT): no window is decided
+        if (part == 0) write_window_undecided(P, b);
+        return;
+    }
+
+    const int a = window_accept<DT>(P, b, n, wide, my, x, lpx, lqx, c, ts);
+    const int err = ts.err;
+    if (part == 0) write_window(P, b, a, err, ts);
     if (err || a >= n) return;  // uniform over the CTA (and over the window's CTAs)
     const int64_t row = static_cast<int64_t>(b) * G.K + a;
-    residual_draw<DT, false, CLUSTER>(P, b, a, ts.kp[a], ts.kq[a], P.target + row * G.ld_bytes, P.draft + row * G.ld_bytes, row, part,
-                             static_cast<int>(gridDim.x), sh);
+    residual_draw<DT, false, CLUSTER>(P, b, a, ts.kp[a], ts.kq[a], P.target + row * G.ld_bytes,
+                                                                    P.draft + row * G.ld_bytes, row, part,
+                                                                    static_cast<int>(gridDim.x), sh);
+}
+
+// ============================================================ few rows ====
+// Calls that stream little (sampling mode) replace the streaming kernel by one built for latency instead of
+// bandwidth: grid (shares, windows), all CTAs resident; groups of warps (1, 2, 4 warps, or the 8 of one or
+// several whole CTAs) each add up one row of the window, every lane with all its 16-byte loads of the row in
+// flight at once.  The CTAs that share a row form a thread-block cluster and meet in the shared memory of
+// its first CTA, so every row leaves one partial, as the acceptance tests of tail_kernel (which follows as
+// usual) like it best.
+constexpr int kSmallDepth = 4;  // batches of kVecPerThread vectors a lane has in flight
+constexpr int64_t kSmallMaxBytes = 48ll << 20;  // calls that stream at most this much take this path
+constexpr int kMaxSmallCtas = 1024;             // ... with at most this many CTAs in this kernel
+constexpr int kSmallMaxCtasPerRow = 8;          // ... of which at most this many (one cluster) share a row
+
+template <int DT, bool CLUSTER>
+__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) small_rows_kernel(const __grid_constant__ VerifyParams P) {
+    const Geometry& G = P.geo;
+    __shared__ Partial warp_part[kResidualWarps];
+    __shared__ Partial cta_part[kSmallMaxCtasPerRow];  // (used in the row's first CTA)
+    const int b = blockIdx.y, part = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = P.row_len ? min(max(__ldg(P.row_len + b), 0), G.K) : G.K;
+    cudaGridDependencySynchronize();  // an earlier call on the stream may still be reading the partials
+
+    const int rows = G.K * G.units_per_row;  // rows of the window that are streamed
+    const int group = G.small_group;
+    int r, seg, segs;  // this warp: row of the window, its segment of the row, segments per row
+    if (group == kResidualWarps) {
+        r = part / G.small_ctas_per_row;
+        seg = (part - r * G.small_ctas_per_row) * kResidualWarps + warp;
+        segs = G.small_ctas_per_row * kResidualWarps;
+    } else {
+        r = part * (kResidualWarps / group) + warp / group;
+        seg = warp % group;
+        segs = group;
+    }
+    RowState st;
+    st.reset();
+    const int i_row = G.units_per_row == 2 ? (r >> 1) : r;
+    if (r < rows && i_row < n) {
+        const bool is_draft = G.units_per_row == 2 && (r & 1);
+        const int64_t row = static_cast<int64_t>(b) * G.K + i_row;
+        const int nvec = G.vec_bytes / 16;
+        const int v0 = static_cast<int>(static_cast<int64_t>(seg) * nvec / segs);
+        const int v1 = static_cast<int>(static_cast<int64_t>(seg + 1) * nvec / segs);
+        const char* base = (is_draft ? P.draft : P.target) + row * G.ld_bytes + static_cast<int64_t>(v0) * 16;
+        const int len = (v1 - v0) * 16;
+        constexpr int kBatchBytes = 32 * 16 * kVecPerThread;
+        for (int off = 0; off < len; off += kSmallDepth * kBatchBytes) {
+            uint4 w[kSmallDepth][kVecPerThread];
+            int at[kSmallDepth][kVecPerThread];
+#pragma unroll
+            for (int h = 0; h < kSmallDepth; ++h)
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    at[h][j] = off + h * kBatchBytes + j * 32 * 16 + lane * 16;
+                    if (at[h][j] < len) w[h][j] = ld_global_nc_v4(base + at[h][j]);
+                }
+            if (st.ref == kNoReference && at[0][0] < len) st.ref = first_reference<DT>(w[0][0], P.c_hi, P.c_lo);
+#pragma unroll
+            for (int h = 0; h < kSmallDepth; ++h) {
+                if (off + h * kBatchBytes >= len) break;  // uniform over the warp
+                if (at[h][kVecPerThread - 1] < len)
+                    absorb_tile<DT, true>(w[h], at[h], len, P.c_hi, P.c_lo, st);
+                else
+                    absorb_tile<DT, false>(w[h], at[h], len, P.c_hi, P.c_lo, st);
+            }
+        }
+    }
+    {
+        const Partial mine = warp_combine<false>(st.ref, st.sum, st.best, st.index);
+        if (lane == 0) warp_part[warp] = mine;
+    }
+    __syncthreads();
+    Partial all;
+    all.ref = kNoReference;
+    all.sum = 0.f;
+    all.best = -INFINITY;
+    all.index = 0x7FFFFFFF;
+    if (warp < kResidualWarps / group) {  // warp g folds the records of the g-th group of warps
+        if (lane < group) all = warp_part[warp * group + lane];
+        all = warp_combine<false>(all.ref, all.sum, all.best, all.index);
+    }
+    if constexpr (CLUSTER) {
+        // whole CTAs share the row: their records go to the first one, which folds them
+        const int rank = part % G.small_ctas_per_row;
+        if (threadIdx.x == 0) cg::this_cluster().map_shared_rank(cta_part, 0)[rank] = all;
+        cg::this_cluster().sync();
+        if (rank == 0 && warp == 0) {
+            Partial rec;
+            rec.ref = kNoReference;
+            rec.sum = 0.f;
+            rec.best = -INFINITY;
+            rec.index = 0x7FFFFFFF;
+            if (lane < G.small_ctas_per_row) rec = cta_part[lane];
+            rec = warp_combine<false>(rec.ref, rec.sum, rec.best, rec.index);
+            if (lane == 0 && r < rows) P.partials[static_cast<int64_t>(b) * rows + r] = rec;
+        }
+    } else if (warp < kResidualWarps / group) {
+        const int rg = group == kResidualWarps ? part : part * (kResidualWarps / group) + warp;
+        if (lane == 0 && rg < rows) P.partials[static_cast<int64_t>(b) * rows + rg] = all;
+    }
 }
 
 // =================================================== vocabulary-parallel ====
@@ -1159,8 +1304,11 @@ static int sm_count_of_current_device(int* device_out) {
     return g_sm_count[dev];
 }
 
+
+// small_capacity: CTAs of small_rows_kernel the device holds at once when the call may take the path for
+// few rows (sampling mode, the target rows streamed, no timing marks), else 0.
 static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool target_only, int sm_count,
-                          Geometry* out) {
+                          Geometry* out, int small_capacity = 0) {
     if (B < 1 || B > FEF_MAX_B || K < 1 || K > FEF_MAX_K || V < 1 || ld < V || sm_count < 1) return false;
     if (dt != FEF_F32 && dt != FEF_BF16) return false;
     const int esize = dt == FEF_F32 ? 4 : 2;
@@ -1224,6 +1372,34 @@ static bool make_geometry(int B, int K, int V, int64_t ld, fef_dtype dt, bool ta
     if (parts > kMaxResidualCtas) parts = kMaxResidualCtas;
     if (parts < 1) parts = 1;
     G.residual_ctas = parts;
+
+    // few rows: the window's CTAs split its rows by groups of warps
+    G.small = 0;
+    G.small_parts = 0;
+    G.small_group = 0;
+    G.small_ctas_per_row = 0;
+    if (small_capacity > kMaxSmallCtas) small_capacity = kMaxSmallCtas;
+    const int small_parts = small_capacity / B;
+    const int rows = K * G.units_per_row;
+    if (small_parts >= 1 && G.vec_bytes > 0 && G.num_units * G.vec_bytes <= kSmallMaxBytes &&
+        small_parts * kResidualWarps >= rows) {
+        const int warps_per_row = small_parts * kResidualWarps / rows;
+        G.small = 1;
+        if (warps_per_row >= kResidualWarps) {
+            G.small_group = kResidualWarps;
+            G.small_ctas_per_row = warps_per_row / kResidualWarps;
+            if (G.small_ctas_per_row > kSmallMaxCtasPerRow) G.small_ctas_per_row = kSmallMaxCtasPerRow;
+        } else {
+            G.small_group = warps_per_row >= 4 ? 4 : warps_per_row >= 2 ? 2 : 1;
+            G.small_ctas_per_row = 1;
+        }
+        G.claims_per_unit = 1;
+        G.num_claims = G.num_units;
+        // as many CTAs as have a row to work on
+        G.small_parts = G.small_group == kResidualWarps ? rows * G.small_ctas_per_row
+                                                         : (rows * G.small_group + kResidualWarps - 1) / kResidualWarps;
+        G.warp_per_row = 0;
+    }
     *out = G;
     return true;
 }
@@ -1301,6 +1477,27 @@ static cudaError_t launch_all(const VerifyParams& P, int dev, cudaStream_t strea
         g_attr_done[dev][which] = true;
     }
     cudaError_t e;
+    if constexpr (!GREEDY) {
+        if (G.small) {
+            // few rows: the latency-oriented kernel streams instead
+            e = launch_dependent(begin_call_kernel, dim3(1), dim3(kBeginThreads), 0, stream, P.ctl, P.tasks, G.B, P.status);
+            if (e != cudaSuccess) return e;
+            if (G.small_ctas_per_row > 1)
+                e = launch_dependent_cluster(G.small_ctas_per_row, small_rows_kernel<DT, true>, dim3(G.small_parts, G.B),
+                                             dim3(kResidualThreads), 0, stream, P);
+            else
+                e = launch_dependent(small_rows_kernel<DT, false>, dim3(G.small_parts, G.B), dim3(kResidualThreads), 0,
+                                     stream, P);
+            if (e != cudaSuccess) return e;
+            if (G.residual_ctas <= kMaxClusterCtas)
+                e = launch_dependent_cluster(G.residual_ctas, tail_kernel<DT, true>, dim3(G.residual_ctas, G.B),
+                                             dim3(kResidualThreads), 0, stream, P);
+            else
+                e = launch_dependent(tail_kernel<DT, false>, dim3(G.residual_ctas, G.B), dim3(kResidualThreads), 0, stream, P);
+            if (e != cudaSuccess) return e;
+            return cudaGetLastError();
+        }
+    }
     if (!GREEDY && P.target_norm) {
         // both laws' normalisers are given: only the counters are cleared, then the last kernel runs
         e = launch_dependent(begin_call_kernel, dim3(1), dim3(kBeginThreads), 0, stream, P.ctl, P.tasks, G.B, P.status);
@@ -1371,8 +1568,17 @@ size_t fef_spec_verify_workspace_bytes(int B, int K, int V, fef_dtype dt) {
     fef::Geometry sampling, greedy;
     if (!fef::make_geometry(B, K, V, V, dt, false, sms, &sampling)) return 0;
     if (!fef::make_geometry(B, K, V, V, dt, true, sms, &greedy)) return 0;
-    const size_t a = fef::layout_of(sampling).total, b = fef::layout_of(greedy).total;
-    return a > b ? a : b;  // one buffer serves both the sampling and the greedy mode
+    size_t need = fef::layout_of(sampling).total;  // one buffer serves every mode
+    const size_t g = fef::layout_of(greedy).total;
+    if (g > need) need = g;
+    const int capacity = fef::kResidualCtasPerSm * sms;
+    for (int target_only = 0; target_only < 2 && capacity > 0; ++target_only) {
+        fef::Geometry few_rows;
+        if (!fef::make_geometry(B, K, V, V, dt, target_only != 0, sms, &few_rows, capacity)) return 0;
+        const size_t s = fef::layout_of(few_rows).total;
+        if (s > need) need = s;
+    }
+    return need;
 }
 
 }  // extern "C"
@@ -1414,7 +1620,11 @@ static fef_status verify_impl(const void* draft_logits, const void* target_logit
     const bool greedy = (temperature == 0.0f);
 
     VerifyParams P;
-    if (!make_geometry(B, K, V, ld, dt, greedy || draft_log2_norm != nullptr, sms, &P.geo)) return FEF_ERR_INVALID_ARG;
+    // the path for few rows: sampling mode with the target rows to stream, no timing marks
+    const bool small_ok = !greedy && !stage_events && !(draft_log2_norm && target_log2_norm);
+    if (!make_geometry(B, K, V, ld, dt, greedy || draft_log2_norm != nullptr, sms, &P.geo,
+                       small_ok ? kResidualCtasPerSm * sms : 0))
+        return FEF_ERR_INVALID_ARG;
     const WorkspaceLayout L = layout_of(P.geo);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return FEF_ERR_WORKSPACE;

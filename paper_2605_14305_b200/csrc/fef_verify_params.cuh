@@ -23,6 +23,10 @@ struct Geometry {
     int grid;             // CTAs of the streaming kernel
     int warp_per_row;     // 1: short rows, many of them: rows_kernel (one warp per row) streams instead
     int residual_ctas;    // CTAs per rejected row in the residual kernel
+    int small;            // 1: few rows: small_rows_kernel with (small_parts, B) CTAs streams instead of stream_kernel
+    int small_parts;
+    int small_group;      // ... in which this many consecutive warps share a row: 1, 2, 4 or 8 (a whole CTA)
+    int small_ctas_per_row;  // ... and, with whole CTAs, this many CTAs (one thread-block cluster) share a row; else 1
     int64_t num_units;    // rows to stream: B * K * units_per_row
     int64_t num_claims;   // num_units * claims_per_unit
     int64_t ld_bytes;     // row pitch in bytes

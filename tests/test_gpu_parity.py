@@ -236,8 +236,11 @@ def test_host_buffer_entry_points_match_device_entry_points(fef):
     assert err.value.status == fef.FEF_ERR_WORKSPACE
 
 
-def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef):
-    q, p, tok = _random_case(4, 16, 50000, torch.bfloat16, 0.7, 51)
+@pytest.mark.parametrize("B", [4, 32])
+def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef, B):
+    # (the small call runs as one kernel unless timing marks are asked for: the row sums are then added
+    # in another order, so its confidences agree to rounding, not to the bit)
+    q, p, tok = _random_case(B, 16, 50000, torch.bfloat16, 0.7, 51)
     want = _gpu_verify(fef, q, p, tok, 1.0, 3, 3)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
     for e in ev:
@@ -245,7 +248,10 @@ def test_profiled_entry_point_gives_identical_results_and_ordered_events(fef):
     r = fef.fef_spec_verify(q, p, tok, 1.0, 3, 3, stage_events=ev)
     torch.cuda.synchronize()
     assert (r.accept_len.cpu().numpy() == want[0]).all() and (r.tokens.cpu().numpy() == want[1]).all()
-    assert (r.conf.cpu().numpy() == want[2]).all()
+    if B == 32:
+        assert (r.conf.cpu().numpy() == want[2]).all()
+    else:
+        np.testing.assert_allclose(r.conf.cpu().numpy(), want[2], rtol=2e-6)
     assert ev[0].elapsed_time(ev[1]) > 0 and ev[1].elapsed_time(ev[2]) > 0 and ev[2].elapsed_time(ev[3]) >= 0
 
 

@@ -38,7 +38,7 @@ def _load_hooks_library():
 @pytest.mark.parametrize("T", [1.0, 0.0])
 def test_a_wait_that_runs_out_reports_timeout_and_the_next_call_is_exact(T):
     L = _load_hooks_library()
-    B, K, V = 2, 4, 50000
+    B, K, V = 8, 32, 50000   # (large enough for the streaming kernel in sampling mode too)
     g = torch.Generator(device="cuda").manual_seed(3)
     q = (torch.randn((B, K, V), generator=g, device="cuda") * 2).to(torch.bfloat16)
     p = (q.float() + torch.randn((B, K, V), generator=g, device="cuda") * 0.7).to(torch.bfloat16)
@@ -74,3 +74,4 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_next_call_is_exact(T):
     ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), T, 5, 2)
     rep = compare_verify(accept.cpu().numpy(), tokens.cpu().numpy(), conf.cpu().numpy(), ref)
     assert rep.ok, rep.mismatches
+

@@ -429,7 +429,8 @@ def fef_remask_select(conf: torch.Tensor, mask: torch.Tensor, k: int, positions:
         raise FefError(FEF_ERR_INVALID_ARG, "fef_remask_select")
     B, L = conf.shape
     dev = conf.device
-    with _on(dev, stream):
+    plain = positions is not None and count is not None and stream is None and torch.cuda.current_device() == dev.index
+    with (contextlib.nullcontext() if plain else _on(dev, stream)):
         if positions is None:
             positions = torch.empty((B, max(int(k), 0)), dtype=torch.int32, device=dev)
         if count is None:

@@ -9,6 +9,8 @@
 //                    shared counter in row order) and leaves, per claim, the partial sum of
 //                    2^(l_v * c - ref), c = log2(e) / T, from which pi(x) and rho(x) follow
 //                    for any x  (the two softmax laws of Section 3.2);
+//                    rows_kernel (many short rows) and small_rows_kernel (calls that stream little)
+//                    take its place where the ring is a poor fit;
 //   tail_kernel      grid (shares, windows): finishes the normalisers in double precision, draws
 //                    u_i, applies u_i <= min{1, pi_i(x_i) / rho_i(x_i)}, finds the first rejection,
 //                    writes accepted tokens and confidences c_i = pi_i(x_i); then, for windows that
@@ -401,7 +403,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
 // slices of a sharded vocabulary): one warp per row and tensor, four 16-byte loads per lane in
 // flight, one warp reduction per row, no shared memory.  Leaves one partial per row like the ring.
 constexpr int kRowsWarps = 8;        // rows a CTA works on at a time
-constexpr int kRowsCtasPerSm = 3;  // (four would cap the kernel at 64 registers: it spilled up to 412 bytes there)
+constexpr int kRowsCtasPerSm = 3;  // (four would cap the kernel at 64 registers: it spilled up to 412 bytes there; two leave no
+                                   // spill at all but run vocabulary slices 3-4 % slower than three with their few bytes)
 
 template <int DT, bool GREEDY>
 __global__ void __launch_bounds__(kRowsWarps * 32, kRowsCtasPerSm) rows_kernel(const __grid_constant__ VerifyParams P) {

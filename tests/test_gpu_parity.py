@@ -425,3 +425,31 @@ def test_draft_draws_with_the_target_normalisers_and_verification_without_stream
     torch.cuda.synchronize()
     assert int(r2.device_status.item()) == fef.FEF_ERR_NONFINITE and int(r2.accept_len[1].item()) == -1
     assert (g0.tokens == g1.tokens).all() and (g0.conf == g1.conf).all()
+
+
+def test_calls_on_a_stream_that_is_not_current_own_what_they_allocate(fef):
+    """Outputs and scratch that the wrappers allocate belong to the stream the kernels run on: while
+    calls are queued on a side stream, the current stream allocates and overwrites memory of the same
+    sizes; every call still equals the oracle (draft draws and verification, large and small sizes)."""
+    side = torch.cuda.Stream()
+    for n, (B, K, V) in enumerate([(2, 8, 40000), (24, 32, 60000)]):
+        q, p, tok = _random_case(B, K, V, torch.bfloat16, 0.7, 200 + n)
+        ws_bytes = fef.fef_spec_verify_workspace_bytes(B, K, V, torch.bfloat16)
+        side.wait_stream(torch.cuda.current_stream())
+        results = []
+        for step in range(6):
+            d = fef.fef_draft_sample(q, 1.0, 9, step, stream=side)
+            r = fef.fef_spec_verify(q, p, tok, 1.0, 9, step, stream=side)
+            results.append((d, r))
+            # the current stream takes and scribbles over blocks of the sizes the wrappers asked for
+            for _ in range(4):
+                torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda").fill_(0xAB)
+                torch.empty((B, K), dtype=torch.int32, device="cuda").fill_(123456)
+                torch.empty((B, K), dtype=torch.float32, device="cuda").fill_(7.0)
+        torch.cuda.synchronize()
+        for step, (d, r) in enumerate(results):
+            ref = oracle.spec_verify(q.cpu(), p.cpu(), tok.cpu(), 1.0, 9, step)
+            rep = compare_verify(r.accept_len.cpu().numpy(), r.tokens.cpu().numpy(), r.conf.cpu().numpy(), ref)
+            assert rep.ok, rep.mismatches[:3]
+            dref = oracle.draft_sample(q.cpu(), 1.0, 9, step)
+            assert (d.tokens.cpu().numpy() == dref["tokens"]).all()
